@@ -1,0 +1,167 @@
+/*
+ * ptq_linear.h -- C ABI of the B200 (sm_100a) PTS W8A8 linear layer.
+ *
+ * The operation is the quantized linear layer of PTQ4VM (arXiv 2412.20386),
+ * Sec. 5.1 "Per-Token Static (PTS) Quantization":
+ *
+ *      Y  ~=  diag(Delta_W) . (W-bar . X-bar) . diag(Delta_X)
+ *
+ * with the SmoothQuant scale s of Sec. 2.4 (Eq. smooth_scale, Eq. smooth)
+ * applied to the activations on the fly and assumed already folded into the
+ * integer weight.  Written row-major, for token row m = b*T + t:
+ *
+ *   Q1  q[m,k]   = clamp( rne( (x[m,k] / s[k]) / dx[t] ), -128, 127 )      int8
+ *   G1  acc[m,n] = sum_k q[m,k] * Wq[n,k]                                  int32
+ *   E1  y[m,n]   = fp16( float(acc[m,n]) * dx[t] * dw[n] + bias[n] )       fp16
+ *
+ * Q1 uses two IEEE binary32 divisions in that order, round-to-nearest-even,
+ * NaN -> 0, +-inf -> 127 / -128.  G1 is exact.  E1 is evaluated in binary32.
+ * The four parts named in Appendix B.1 of the paper (activation smoothing,
+ * quantization, integer GEMM, dequantization) map to Q1 (first two), G1, E1.
+ *
+ * Conventions
+ *   - "host" / "device" in a parameter comment says where the pointer lives.
+ *   - Every function returns a ptq_status_t; none throws, aborts or traps.
+ *     ptq_last_error() gives a thread-local text for the last failure.
+ *   - ptq_linear_create copies all parameters: the caller keeps its arrays.
+ *   - The forward calls allocate nothing, enqueue work on the caller's stream
+ *     and return without synchronising.  A handle is immutable after create,
+ *     so concurrent forwards on different streams are allowed as long as they
+ *     use different workspaces (each handle also carries one device status
+ *     word that all its launches may set; see ptq_linear_device_status).
+ *   - Requires a device of compute capability 10.0 (sm_100a); create fails
+ *     with PTQ_ERR_ARCH elsewhere.  There is no CPU or generic-GPU fallback.
+ */
+#ifndef PTQ_LINEAR_H_
+#define PTQ_LINEAR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ptq_linear ptq_linear_t;   /* opaque; owns device copies of all parameters */
+
+typedef enum {
+    PTQ_OK          = 0,
+    PTQ_ERR_NULL    = 1,   /* a required pointer is NULL */
+    PTQ_ERR_SHAPE   = 2,   /* a dimension is out of range, or the workspace is too small */
+    PTQ_ERR_VALUE   = 3,   /* a parameter value is invalid (non-positive or non-finite step, weight code -128) */
+    PTQ_ERR_ALIGN   = 4,   /* a device pointer is not aligned as required */
+    PTQ_ERR_ARCH    = 5,   /* current device is not compute capability 10.0 */
+    PTQ_ERR_CUDA    = 6,   /* a CUDA runtime / driver call failed; text in ptq_last_error() */
+    PTQ_ERR_NOMEM   = 7,   /* device or host allocation failed (create / calibrate only) */
+    PTQ_ERR_TIMEOUT = 8    /* a bounded device-side wait gave up (reported by ptq_linear_device_status) */
+} ptq_status_t;
+
+/* Flags for create / forward. */
+#define PTQ_FLAG_NONE            0u
+#define PTQ_FLAG_FUSED_PROLOGUE  1u   /* F1: quantize inside the GEMM kernel; no int8 round trip, no workspace */
+
+/* Limits (create returns PTQ_ERR_SHAPE beyond them). */
+#define PTQ_MAX_K   8192
+#define PTQ_MAX_N   65536
+#define PTQ_MAX_T   1048576
+
+/*
+ * Create a layer (Sec. 5.1; weight format of Sec. 2.3).
+ *   K, N, T      input channels D_in, output channels D_out, token positions L per image
+ *   w_q          host, [N,K] row-major int8, the folded integer weight W-bar = quant(W diag(s));
+ *                values in [-127,127] (symmetric range of Sec. 2.3; -128 is rejected)
+ *   w_step       host, [N] fp32, Delta_W per output channel, finite and > 0
+ *   smooth       host, [K] fp32, smoothing scale s (Eq. smooth_scale), finite and > 0
+ *   act_step     host, [T] fp32, Delta_X per token position, finite and > 0
+ *   bias         host, [N] fp32 or NULL (added after the scaling, before the fp16 rounding)
+ *   flags        reserved, pass PTQ_FLAG_NONE
+ * The handle is bound to the device that is current at the time of the call.
+ */
+ptq_status_t ptq_linear_create(ptq_linear_t **out, int K, int N, int T,
+                               const int8_t *w_q, const float *w_step,
+                               const float *smooth, const float *act_step,
+                               const float *bias, unsigned flags);
+
+/* Release the handle and its device memory.  NULL is allowed. */
+void ptq_linear_destroy(ptq_linear_t *h);
+
+/*
+ * Bytes of device workspace ptq_linear_forward needs for a batch of B images:
+ * the int8 codes [B*T, Kpad] with Kpad = K rounded up to 16, or 0 with
+ * PTQ_FLAG_FUSED_PROLOGUE.  Returns 0 for a NULL handle or B < 1.
+ */
+size_t ptq_linear_workspace_bytes(const ptq_linear_t *h, int B, unsigned flags);
+
+/*
+ * Forward pass Q1 -> G1 -> E1 (Sec. 5.1; Appendix B.1).
+ *   x_fp16     device, [B,T,K] contiguous binary16, 2-byte aligned (16-byte alignment and K % 8 == 0
+ *              enable the vectorised load path)
+ *   y_fp16     device, [B,T,N] contiguous binary16; must not overlap x or the workspace
+ *   workspace  device, at least ptq_linear_workspace_bytes(h,B,flags) bytes, 16-byte aligned;
+ *              contents are scratch.  May be NULL with PTQ_FLAG_FUSED_PROLOGUE.
+ *   flags      PTQ_FLAG_NONE: quantize kernel, then GEMM+dequant kernel.
+ *              PTQ_FLAG_FUSED_PROLOGUE: one kernel; same results bit for bit.  Layers whose shape the
+ *              fused kernel does not cover fall back to the two-kernel path and then need the workspace
+ *              (ptq_linear_fused_supported tells which).
+ *   stream     cudaStream_t cast to void* (NULL = legacy default stream)
+ */
+ptq_status_t ptq_linear_forward(const ptq_linear_t *h, const void *x_fp16, int B,
+                                void *y_fp16, void *workspace, size_t workspace_bytes,
+                                unsigned flags, void *stream);
+
+/* 1 if PTQ_FLAG_FUSED_PROLOGUE runs the single fused kernel for this layer, 0 if it falls back. */
+int ptq_linear_fused_supported(const ptq_linear_t *h);
+
+/*
+ * Q1 alone (Appendix B.1, parts 1-2): q_int8 device [B,T,K] dense int8 codes.
+ */
+ptq_status_t ptq_quantize(const ptq_linear_t *h, const void *x_fp16, int B,
+                          void *q_int8, void *stream);
+
+/*
+ * Forward pass with parity taps.  Same as ptq_linear_forward, and additionally writes
+ *   q_int8_out     device, [B,T,K] dense int8 codes of Q1, or NULL
+ *                  (with PTQ_FLAG_FUSED_PROLOGUE the codes never exist in memory; they are then
+ *                  produced by a separate run of the quantize kernel)
+ *   acc_int32_out  device, [B,T,N] dense int32 accumulators of G1, or NULL
+ * The workspace is required unless PTQ_FLAG_FUSED_PROLOGUE is set and q_int8_out is NULL.
+ */
+ptq_status_t ptq_linear_forward_debug(const ptq_linear_t *h, const void *x_fp16, int B,
+                                      void *y_fp16, void *q_int8_out, void *acc_int32_out,
+                                      void *workspace, size_t workspace_bytes,
+                                      unsigned flags, void *stream);
+
+/*
+ * Q0: min-max calibration of the static parameters from a calibration batch
+ * (Eq. smooth_scale with the given integer weights; PTS steps of Sec. 5.1 from
+ * the min-max range of Sec. 2.3):
+ *   maxX[k] = max |xcal[:,:,k]|,  maxW[k] = max_n |w_q[n,k]| * w_step[n]
+ *   s[k]    = sqrt( max(maxX[k],1e-5) / max(maxW[k],1e-5) )
+ *   dx[t]   = max( max_{b,k} |xcal[b,t,k] / s[k]|, 1e-5 ) / 127
+ * all in binary32 with correctly rounded operations, so the result is unique.
+ *   xcal_fp16     device, [Bc,T,K] contiguous binary16
+ *   w_q, w_step   host
+ *   smooth_out    host, [K];  act_step_out  host, [T]
+ * Allocates temporary device memory and synchronises the stream before returning.
+ */
+ptq_status_t ptq_calibrate(int K, int N, int T, const void *xcal_fp16, int Bc,
+                           const int8_t *w_q, const float *w_step,
+                           float *smooth_out, float *act_step_out, void *stream);
+
+/*
+ * Read and clear the handle's device status word.  Synchronises the device.  Returns PTQ_OK, or
+ * PTQ_ERR_TIMEOUT if a kernel launched with this handle abandoned a bounded wait since the last
+ * call (its output is then undefined), or PTQ_ERR_CUDA.
+ */
+ptq_status_t ptq_linear_device_status(const ptq_linear_t *h);
+
+/* Number of kernels this library has launched in the calling process (all handles, all threads). */
+unsigned long long ptq_kernel_launch_count(void);
+
+const char *ptq_status_string(ptq_status_t st);
+const char *ptq_last_error(void);   /* thread-local; valid until the next failing call on this thread */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PTQ_LINEAR_H_ */

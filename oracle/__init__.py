@@ -1,0 +1,181 @@
+"""ctypes binding of the CPU oracle (``ptq_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY.  The oracle is the independent, slow CPU statement of
+what the PTS W8A8 linear layer of PTQ4VM computes (Sec. 5.1, Eq. smooth_scale,
+Eq. smooth).  Only the tests, the smoke check and the CPU-baseline leg of the
+benchmark may import this package; the product package never does, and this
+package imports nothing from the product.
+
+Arrays are numpy: fp16 tensors travel as ``float16`` (viewed as ``uint16`` at
+the C boundary), codes as ``int8``, accumulators as ``int32``.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "ptq_oracle.c")
+_OUT_DIR = os.path.join(_HERE, "_build")
+_SO = os.path.join(_OUT_DIR, "libptq_oracle.so")
+
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile ``ptq_oracle.c`` with gcc (no fast-math, no FMA contraction)."""
+    os.makedirs(_OUT_DIR, exist_ok=True)
+    if (not force and os.path.exists(_SO)
+            and os.path.getmtime(_SO) >= os.path.getmtime(_SRC)):
+        return _SO
+    tmp = _SO + ".tmp.%d" % os.getpid()
+    cmd = ["gcc", "-O2", "-fopenmp", "-ffp-contract=off", "-fno-fast-math",
+           "-std=c99", "-D_DEFAULT_SOURCE", "-Wall", "-shared", "-fPIC", _SRC,
+           "-o", tmp, "-lm"]
+    subprocess.run(cmd, check=True)
+    os.replace(tmp, _SO)
+    return _SO
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is not None:
+        return _lib
+    L = ctypes.CDLL(build())
+    c_long, c_int, vp = ctypes.c_long, ctypes.c_int, ctypes.c_void_p
+    L.ptqo_num_threads.restype = c_int
+    L.ptqo_half_to_float.restype = ctypes.c_float
+    L.ptqo_half_to_float.argtypes = [ctypes.c_uint16]
+    L.ptqo_double_to_half.restype = ctypes.c_uint16
+    L.ptqo_double_to_half.argtypes = [ctypes.c_double]
+    L.ptqo_quantize_one.restype = ctypes.c_int8
+    L.ptqo_quantize_one.argtypes = [ctypes.c_uint16, ctypes.c_float, ctypes.c_float]
+    L.ptqo_quantize.restype = None
+    L.ptqo_quantize.argtypes = [vp, c_long, c_int, c_int, vp, vp, vp]
+    L.ptqo_int_matmul.restype = c_int
+    L.ptqo_int_matmul.argtypes = [vp, vp, c_long, c_int, c_int, vp]
+    L.ptqo_dequant.restype = None
+    L.ptqo_dequant.argtypes = [vp, c_long, c_int, c_int, vp, vp, vp, vp]
+    L.ptqo_linear_forward_rows.restype = c_int
+    L.ptqo_linear_forward_rows.argtypes = [vp, c_long, c_long, c_int, c_int, c_int,
+                                           vp, vp, vp, vp, vp, vp, vp, vp]
+    L.ptqo_calibrate.restype = None
+    L.ptqo_calibrate.argtypes = [vp, c_int, c_int, c_int, vp, vp, c_int, vp, vp]
+    _lib = L
+    return L
+
+
+def _p(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _c(a, dtype):
+    a = np.ascontiguousarray(a)
+    if a.dtype != dtype:
+        raise TypeError("expected %s, got %s" % (np.dtype(dtype), a.dtype))
+    return a
+
+
+def num_threads() -> int:
+    return int(lib().ptqo_num_threads())
+
+
+def half_to_float(bits: int) -> float:
+    return float(lib().ptqo_half_to_float(int(bits)))
+
+
+def double_to_half_bits(v: float) -> int:
+    return int(lib().ptqo_double_to_half(float(v)))
+
+
+def quantize_one(x_bits: int, s: float, dx: float) -> int:
+    return int(lib().ptqo_quantize_one(int(x_bits), float(s), float(dx)))
+
+
+def quantize(x, T, s, dx):
+    """Q1: x fp16 [M,K] -> int8 codes [M,K]; s fp32 [K]; dx fp32 [T]."""
+    x = _c(x, np.float16)
+    M, K = x.shape
+    s = _c(s, np.float32)
+    dx = _c(dx, np.float32)
+    assert s.shape == (K,) and dx.shape == (T,)
+    q = np.empty((M, K), np.int8)
+    lib().ptqo_quantize(_p(x), M, K, T, _p(s), _p(dx), _p(q))
+    return q
+
+
+def int_matmul(q, wq):
+    """G1: q int8 [M,K] x wq int8 [N,K]^T -> int32 [M,N] (raises on int32 overflow)."""
+    q = _c(q, np.int8)
+    wq = _c(wq, np.int8)
+    M, K = q.shape
+    N, K2 = wq.shape
+    assert K == K2
+    acc = np.empty((M, N), np.int32)
+    if lib().ptqo_int_matmul(_p(q), _p(wq), M, K, N, _p(acc)):
+        raise OverflowError("accumulator does not fit in int32")
+    return acc
+
+
+def dequant(acc, T, dx, dw, bias=None):
+    """E1: int32 [M,N] -> fp16 [M,N] = acc * dx[m mod T] * dw[n] (+ bias[n])."""
+    acc = _c(acc, np.int32)
+    M, N = acc.shape
+    dx = _c(dx, np.float32)
+    dw = _c(dw, np.float32)
+    if bias is not None:
+        bias = _c(bias, np.float32)
+        assert bias.shape == (N,)
+    assert dx.shape == (T,) and dw.shape == (N,)
+    y = np.empty((M, N), np.float16)
+    lib().ptqo_dequant(_p(acc), M, N, T, _p(dx), _p(dw), _p(bias), _p(y))
+    return y
+
+
+def linear_forward(x, T, wq, dw, s, dx, bias=None, rows=None, taps=False):
+    """Whole path Q1 -> G1 -> E1 on rows [m0, m1) of x fp16 [M,K].
+
+    Returns y fp16 [m1-m0, N], or (y, q, acc) when ``taps`` is set.
+    """
+    x = _c(x, np.float16)
+    M, K = x.shape
+    wq = _c(wq, np.int8)
+    N = wq.shape[0]
+    assert wq.shape == (N, K)
+    dw = _c(dw, np.float32)
+    s = _c(s, np.float32)
+    dx = _c(dx, np.float32)
+    assert dw.shape == (N,) and s.shape == (K,) and dx.shape == (T,)
+    if bias is not None:
+        bias = _c(bias, np.float32)
+        assert bias.shape == (N,)
+    m0, m1 = (0, M) if rows is None else rows
+    assert 0 <= m0 <= m1 <= M
+    R = m1 - m0
+    y = np.empty((R, N), np.float16)
+    q = np.empty((R, K), np.int8) if taps else None
+    acc = np.empty((R, N), np.int32) if taps else None
+    rc = lib().ptqo_linear_forward_rows(_p(x), m0, m1, K, N, T, _p(wq), _p(dw), _p(s),
+                                        _p(dx), _p(bias), _p(y), _p(q), _p(acc))
+    if rc < 0:
+        raise ValueError("K too large for the oracle's row buffer")
+    if rc:
+        raise OverflowError("accumulator does not fit in int32")
+    return (y, q, acc) if taps else y
+
+
+def calibrate(xcal, wq, dw):
+    """Q0: xcal fp16 [Bc,T,K], wq int8 [N,K], dw fp32 [N] -> (s fp32 [K], dx fp32 [T])."""
+    xcal = _c(xcal, np.float16)
+    Bc, T, K = xcal.shape
+    wq = _c(wq, np.int8)
+    N = wq.shape[0]
+    assert wq.shape == (N, K)
+    dw = _c(dw, np.float32)
+    s = np.empty(K, np.float32)
+    dx = np.empty(T, np.float32)
+    lib().ptqo_calibrate(_p(xcal), Bc, T, K, _p(wq), _p(dw), N, _p(s), _p(dx))
+    return s, dx

@@ -1,0 +1,216 @@
+"""ctypes binding of ``libptq_linear.so`` (the C ABI of ``include/ptq_linear.h``).
+
+Argument marshalling only: every step of the path (quantize, integer GEMM,
+dequantize, calibration reductions) runs in the library's CUDA kernels.  torch
+tensors are used for device memory and streams; their ``data_ptr()`` crosses
+the boundary as a plain pointer.  There is no fallback: if the library is
+missing, loading raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SO = os.path.join(_HERE, "libptq_linear.so")
+
+FLAG_NONE = 0
+FLAG_FUSED_PROLOGUE = 1
+
+_STATUS_NAMES = {0: "PTQ_OK", 1: "PTQ_ERR_NULL", 2: "PTQ_ERR_SHAPE", 3: "PTQ_ERR_VALUE",
+                 4: "PTQ_ERR_ALIGN", 5: "PTQ_ERR_ARCH", 6: "PTQ_ERR_CUDA", 7: "PTQ_ERR_NOMEM",
+                 8: "PTQ_ERR_TIMEOUT"}
+
+_lib = None
+
+
+class PtqError(RuntimeError):
+    def __init__(self, status: int, text: str):
+        super().__init__("%s: %s" % (_STATUS_NAMES.get(status, status), text))
+        self.status = status
+
+
+def library_path() -> str:
+    return _SO
+
+
+def load_library() -> ctypes.CDLL:
+    """Load the shared library (built by ``paper_2412_20386_b200.build``); raise if absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_SO):
+        raise ImportError(
+            "%s not found: build it with `python -m paper_2412_20386_b200.build` "
+            "(nvcc, sm_100a). There is no fallback implementation." % _SO)
+    L = ctypes.CDLL(_SO)
+    vp, ci, cu, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_uint, ctypes.c_size_t
+    L.ptq_linear_create.restype = ci
+    L.ptq_linear_create.argtypes = [ctypes.POINTER(vp), ci, ci, ci, vp, vp, vp, vp, vp, cu]
+    L.ptq_linear_destroy.restype = None
+    L.ptq_linear_destroy.argtypes = [vp]
+    L.ptq_linear_workspace_bytes.restype = sz
+    L.ptq_linear_workspace_bytes.argtypes = [vp, ci, cu]
+    L.ptq_linear_forward.restype = ci
+    L.ptq_linear_forward.argtypes = [vp, vp, ci, vp, vp, sz, cu, vp]
+    L.ptq_linear_fused_supported.restype = ci
+    L.ptq_linear_fused_supported.argtypes = [vp]
+    L.ptq_quantize.restype = ci
+    L.ptq_quantize.argtypes = [vp, vp, ci, vp, vp]
+    L.ptq_linear_forward_debug.restype = ci
+    L.ptq_linear_forward_debug.argtypes = [vp, vp, ci, vp, vp, vp, vp, sz, cu, vp]
+    L.ptq_calibrate.restype = ci
+    L.ptq_calibrate.argtypes = [ci, ci, ci, vp, ci, vp, vp, vp, vp, vp]
+    L.ptq_linear_device_status.restype = ci
+    L.ptq_linear_device_status.argtypes = [vp]
+    L.ptq_kernel_launch_count.restype = ctypes.c_ulonglong
+    L.ptq_kernel_launch_count.argtypes = []
+    L.ptq_status_string.restype = ctypes.c_char_p
+    L.ptq_status_string.argtypes = [ci]
+    L.ptq_last_error.restype = ctypes.c_char_p
+    L.ptq_last_error.argtypes = []
+    _lib = L
+    return L
+
+
+def _check(status: int):
+    if status != 0:
+        raise PtqError(status, load_library().ptq_last_error().decode("utf-8", "replace"))
+
+
+def _host(a, dtype, shape=None):
+    if a is None:
+        return None
+    a = np.ascontiguousarray(a, dtype=dtype)
+    if shape is not None and a.shape != tuple(shape):
+        raise ValueError("expected shape %s, got %s" % (tuple(shape), a.shape))
+    return a
+
+
+def _hp(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _stream_ptr(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(int(stream.cuda_stream))
+
+
+def kernel_launch_count() -> int:
+    return int(load_library().ptq_kernel_launch_count())
+
+
+class PtqLinear:
+    """One PTS W8A8 linear layer on the current CUDA device (``ptq_linear_create``)."""
+
+    def __init__(self, w_q, w_step, smooth, act_step, bias=None, flags: int = 0):
+        L = load_library()
+        w_q = _host(w_q, np.int8)
+        if w_q.ndim != 2:
+            raise ValueError("w_q must be [N,K]")
+        self.N, self.K = int(w_q.shape[0]), int(w_q.shape[1])
+        act_step = _host(act_step, np.float32)
+        self.T = int(act_step.shape[0])
+        w_step = _host(w_step, np.float32, (self.N,))
+        smooth = _host(smooth, np.float32, (self.K,))
+        bias = _host(bias, np.float32, (self.N,))
+        h = ctypes.c_void_p()
+        _check(L.ptq_linear_create(ctypes.byref(h), self.K, self.N, self.T, _hp(w_q), _hp(w_step),
+                                   _hp(smooth), _hp(act_step), _hp(bias), flags))
+        self._h = h
+        self._L = L
+
+    def close(self):
+        if getattr(self, "_h", None):
+            self._L.ptq_linear_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- queries ---------------------------------------------------------------
+    def workspace_bytes(self, B: int, flags: int = 0) -> int:
+        return int(self._L.ptq_linear_workspace_bytes(self._h, int(B), flags))
+
+    def fused_supported(self) -> bool:
+        return bool(self._L.ptq_linear_fused_supported(self._h))
+
+    def device_status(self):
+        _check(self._L.ptq_linear_device_status(self._h))
+
+    # -- calls -----------------------------------------------------------------
+    def _batch(self, x):
+        import torch
+        if x.dtype != torch.float16 or not x.is_cuda or not x.is_contiguous():
+            raise ValueError("x must be a contiguous CUDA float16 tensor")
+        if x.numel() % (self.T * self.K) != 0 or x.shape[-1] != self.K:
+            raise ValueError("x must be [B,T,K] with T=%d K=%d" % (self.T, self.K))
+        return x.numel() // (self.T * self.K)
+
+    def forward(self, x, y=None, workspace=None, flags: int = 0, stream=None):
+        """``ptq_linear_forward``: x fp16 [B,T,K] -> y fp16 [B,T,N] (both on the device)."""
+        import torch
+        B = self._batch(x)
+        if y is None:
+            y = torch.empty((B, self.T, self.N), dtype=torch.float16, device=x.device)
+        need = self.workspace_bytes(B, flags)
+        if workspace is None and need:
+            workspace = torch.empty(need, dtype=torch.uint8, device=x.device)
+        wptr = workspace.data_ptr() if workspace is not None else None
+        wbytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
+        _check(self._L.ptq_linear_forward(self._h, x.data_ptr(), B, y.data_ptr(), wptr, wbytes,
+                                          flags, _stream_ptr(stream)))
+        return y
+
+    def quantize(self, x, q=None, stream=None):
+        """``ptq_quantize``: x fp16 [B,T,K] -> int8 codes [B,T,K]."""
+        import torch
+        B = self._batch(x)
+        if q is None:
+            q = torch.empty((B, self.T, self.K), dtype=torch.int8, device=x.device)
+        _check(self._L.ptq_quantize(self._h, x.data_ptr(), B, q.data_ptr(), _stream_ptr(stream)))
+        return q
+
+    def forward_debug(self, x, flags: int = 0, want_q=True, want_acc=True, stream=None):
+        """``ptq_linear_forward_debug``: returns (y, q or None, acc or None)."""
+        import torch
+        B = self._batch(x)
+        dev = x.device
+        y = torch.empty((B, self.T, self.N), dtype=torch.float16, device=dev)
+        q = torch.empty((B, self.T, self.K), dtype=torch.int8, device=dev) if want_q else None
+        acc = torch.empty((B, self.T, self.N), dtype=torch.int32, device=dev) if want_acc else None
+        need = self.workspace_bytes(B, 0)
+        ws = torch.empty(need, dtype=torch.uint8, device=dev)
+        _check(self._L.ptq_linear_forward_debug(
+            self._h, x.data_ptr(), B, y.data_ptr(),
+            q.data_ptr() if q is not None else None,
+            acc.data_ptr() if acc is not None else None,
+            ws.data_ptr(), need, flags, _stream_ptr(stream)))
+        return y, q, acc
+
+
+def calibrate(xcal, w_q, w_step, stream=None):
+    """``ptq_calibrate``: device fp16 [Bc,T,K] -> (s fp32 [K], dx fp32 [T]) as numpy arrays."""
+    import torch
+    L = load_library()
+    if xcal.dtype != torch.float16 or not xcal.is_cuda or not xcal.is_contiguous() or xcal.dim() != 3:
+        raise ValueError("xcal must be a contiguous CUDA float16 tensor [Bc,T,K]")
+    Bc, T, K = (int(v) for v in xcal.shape)
+    w_q = _host(w_q, np.int8)
+    N = int(w_q.shape[0])
+    if w_q.shape != (N, K):
+        raise ValueError("w_q must be [N,K]")
+    w_step = _host(w_step, np.float32, (N,))
+    s = np.empty(K, np.float32)
+    dx = np.empty(T, np.float32)
+    _check(L.ptq_calibrate(K, N, T, xcal.data_ptr(), Bc, _hp(w_q), _hp(w_step), _hp(s), _hp(dx),
+                           _stream_ptr(stream)))
+    return s, dx
