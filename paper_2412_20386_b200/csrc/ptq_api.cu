@@ -1,0 +1,514 @@
+// Host side of the C ABI declared in include/ptq_linear.h: argument validation, parameter
+// preparation (padding, reciprocals, tensor maps) and kernel launches.  No compute happens here.
+#include "../../include/ptq_linear.h"
+
+#include <cuda.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+#include <new>
+#include <vector>
+
+#include "ptq_calibrate.cuh"
+#include "ptq_gemm.cuh"
+#include "ptq_quantize.cuh"
+
+namespace {
+
+thread_local char g_err[512] = "";
+std::atomic<unsigned long long> g_launches{0};
+
+ptq_status_t fail(ptq_status_t st, const char *fmt, ...)
+{
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+    return st;
+}
+
+#define PTQ_CUDA(call)                                                                         \
+    do {                                                                                       \
+        cudaError_t e_ = (call);                                                               \
+        if (e_ != cudaSuccess)                                                                 \
+            return fail(e_ == cudaErrorMemoryAllocation ? PTQ_ERR_NOMEM : PTQ_ERR_CUDA,        \
+                        "%s failed: %s", #call, cudaGetErrorString(e_));                       \
+    } while (0)
+
+// cuTensorMapEncodeTiled is reached through the runtime's driver entry point query, so the
+// library has no link-time dependency on libcuda and loads on machines without a driver.
+typedef CUresult (*encode_tiled_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                    const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                    CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                    CUtensorMapFloatOOBfill);
+
+encode_tiled_fn get_encode_tiled()
+{
+    static encode_tiled_fn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<encode_tiled_fn>(p);
+    });
+    return fn;
+}
+
+// 2-D row-major tensor [rows, cols] with `pitch_bytes` between rows; box [box_rows, box_cols];
+// 128-byte swizzle (box_cols * elem_bytes must be 128); out-of-range elements read as zero and
+// are skipped on stores.
+ptq_status_t make_map_2d(CUtensorMap *map, CUtensorMapDataType dt, int elem_bytes, const void *ptr,
+                         unsigned long long cols, unsigned long long rows, unsigned long long pitch_bytes,
+                         unsigned box_cols, unsigned box_rows)
+{
+    encode_tiled_fn enc = get_encode_tiled();
+    if (!enc) return fail(PTQ_ERR_CUDA, "cuTensorMapEncodeTiled entry point not available");
+    if (box_cols * elem_bytes != 128 || box_rows == 0 || box_rows > 256)
+        return fail(PTQ_ERR_SHAPE, "internal: bad TMA box %u x %u", box_rows, box_cols);
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {pitch_bytes};
+    cuuint32_t box[2] = {box_cols, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = enc(map, dt, 2, const_cast<void *>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS)
+        return fail(PTQ_ERR_CUDA, "cuTensorMapEncodeTiled failed with CUresult %d (cols %llu rows %llu pitch %llu)",
+                    static_cast<int>(r), cols, rows, pitch_bytes);
+    return PTQ_OK;
+}
+
+inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
+inline int gcd_int(int a, int b) { while (b) { int t = a % b; a = b; b = t; } return a; }
+
+bool ranges_overlap(const void *a, size_t na, const void *b, size_t nb)
+{
+    const uintptr_t a0 = reinterpret_cast<uintptr_t>(a), b0 = reinterpret_cast<uintptr_t>(b);
+    return a0 < b0 + nb && b0 < a0 + na;
+}
+
+}  // namespace
+
+struct ptq_linear {
+    int K = 0, N = 0, T = 0;
+    int Kpad = 0;              // pitch of the codes workspace and of the padded weight: K rounded up to 16
+    int BN = 0, n_tiles = 0;   // GEMM tiling along N
+    int k_blocks = 0, last_mmas = 0;
+    bool fast_div = false;     // all scales inside the range where the reciprocal route is exact
+    int device = -1;
+    int num_sms = 0;
+    int8_t *d_w = nullptr;     // [n_tiles*BN, Kpad], zero padded
+    float *d_dw = nullptr, *d_bias = nullptr;            // [n_tiles*BN rounded up to 64, +64], zero padded
+    float *d_s = nullptr, *d_rs = nullptr;               // [round_up(K,16)]
+    float *d_dx = nullptr, *d_rdx = nullptr;             // [T]
+    unsigned *d_status = nullptr;
+    CUtensorMap tmW;
+};
+
+namespace {
+
+ptq_status_t upload(void **dst, const void *src, size_t bytes, size_t alloc_bytes)
+{
+    PTQ_CUDA(cudaMalloc(dst, alloc_bytes));
+    PTQ_CUDA(cudaMemset(*dst, 0, alloc_bytes));
+    if (bytes) PTQ_CUDA(cudaMemcpy(*dst, src, bytes, cudaMemcpyHostToDevice));
+    return PTQ_OK;
+}
+
+ptq_status_t check_device(const ptq_linear *h)
+{
+    int dev = -1;
+    PTQ_CUDA(cudaGetDevice(&dev));
+    if (dev != h->device)
+        return fail(PTQ_ERR_CUDA, "handle belongs to device %d but device %d is current", h->device, dev);
+    return PTQ_OK;
+}
+
+template <typename Kern>
+ptq_status_t ensure_smem(Kern kern, int bytes)
+{
+    PTQ_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+    return PTQ_OK;
+}
+
+// Q1 launch: codes to `q` with `q_pitch` bytes between rows.
+ptq_status_t launch_quantize(const ptq_linear *h, const void *x, long long M, void *q, int q_pitch,
+                             cudaStream_t stream)
+{
+    ptq::QuantParams p;
+    p.x = static_cast<const __half *>(x);
+    p.q = static_cast<int8_t *>(q);
+    p.s = h->d_s;
+    p.rs = h->d_rs;
+    p.dx = h->d_dx;
+    p.rdx = h->d_rdx;
+    p.M = M;
+    p.K = h->K;
+    p.T = h->T;
+    p.q_pitch = q_pitch;
+    p.rows_per_iter = 0;
+    const bool vec = (h->K % 16 == 0) && (reinterpret_cast<uintptr_t>(x) % 16 == 0) &&
+                     (reinterpret_cast<uintptr_t>(q) % 16 == 0) && (q_pitch % 16 == 0);
+    if (vec) {
+        const int cpr = h->K / 16;
+        const int mult = cpr / gcd_int(cpr, 256);             // grid must make threads a multiple of cpr
+        const long long chunks = M * cpr;
+        long long want = (chunks + 511) / 512;                // two rows per thread per trip
+        const long long cap = static_cast<long long>(h->num_sms) * 6;
+        if (want > cap) want = cap;
+        if (want < 1) want = 1;
+        const int grid = round_up(static_cast<int>(want), mult);
+        p.rows_per_iter = grid * 256 / cpr;
+        if (h->fast_div)
+            ptq::ptq_quantize_vec16_kernel<true><<<grid, 256, 0, stream>>>(p);
+        else
+            ptq::ptq_quantize_vec16_kernel<false><<<grid, 256, 0, stream>>>(p);
+    } else {
+        long long want = (M * h->K + 255) / 256;
+        const long long cap = static_cast<long long>(h->num_sms) * 8;
+        if (want > cap) want = cap;
+        if (want < 1) want = 1;
+        if (h->fast_div)
+            ptq::ptq_quantize_scalar_kernel<true><<<static_cast<int>(want), 256, 0, stream>>>(p);
+        else
+            ptq::ptq_quantize_scalar_kernel<false><<<static_cast<int>(want), 256, 0, stream>>>(p);
+    }
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    PTQ_CUDA(cudaGetLastError());
+    return PTQ_OK;
+}
+
+// G1+E1 launch on codes [M, Kpad] at `codes`.
+ptq_status_t launch_gemm(const ptq_linear *h, const void *codes, long long M, void *y, void *acc_out,
+                         cudaStream_t stream)
+{
+    static std::once_flag once;
+    static ptq_status_t attr_status = PTQ_OK;
+    std::call_once(once, [] {
+        attr_status = ensure_smem(ptq::ptq_gemm_dequant_kernel<false>, ptq::kGemmSmemBytes);
+        if (attr_status == PTQ_OK) attr_status = ensure_smem(ptq::ptq_gemm_dequant_kernel<true>, ptq::kGemmSmemBytes);
+    });
+    if (attr_status != PTQ_OK) return attr_status;
+
+    CUtensorMap tmA, tmY;
+    ptq_status_t st = make_map_2d(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, codes, static_cast<unsigned long long>(h->K),
+                                  static_cast<unsigned long long>(M), static_cast<unsigned long long>(h->Kpad),
+                                  ptq::kBK, ptq::kBM);
+    if (st != PTQ_OK) return st;
+    const bool tma_store = (h->N % 8 == 0) && (reinterpret_cast<uintptr_t>(y) % 16 == 0);
+    if (tma_store) {
+        st = make_map_2d(&tmY, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, y, static_cast<unsigned long long>(h->N),
+                         static_cast<unsigned long long>(M), static_cast<unsigned long long>(h->N) * 2,
+                         ptq::kStoreBoxCols, 32);
+        if (st != PTQ_OK) return st;
+    } else {
+        tmY = h->tmW;   // never dereferenced by the kernel in this mode
+    }
+
+    ptq::GemmParams p;
+    p.M = M;
+    p.N = h->N;
+    p.K = h->K;
+    p.T = h->T;
+    p.BN = h->BN;
+    p.n_tiles = h->n_tiles;
+    p.m_tiles = static_cast<int>((M + ptq::kBM - 1) / ptq::kBM);
+    p.k_blocks = h->k_blocks;
+    p.last_mmas = h->last_mmas;
+    p.dx = h->d_dx;
+    p.dw = h->d_dw;
+    p.bias = h->d_bias;
+    p.y = static_cast<__half *>(y);
+    p.acc_out = static_cast<int32_t *>(acc_out);
+    p.status = h->d_status;
+    p.use_tma_store = tma_store ? 1 : 0;
+    p.y_vec2 = (h->N % 2 == 0 && reinterpret_cast<uintptr_t>(y) % 4 == 0) ? 1 : 0;
+
+    const long long tiles = static_cast<long long>(p.m_tiles) * p.n_tiles;
+    const int grid = static_cast<int>(tiles < h->num_sms ? tiles : h->num_sms);
+    if (acc_out)
+        ptq::ptq_gemm_dequant_kernel<true><<<grid, ptq::kGemmThreads, ptq::kGemmSmemBytes, stream>>>(tmA, h->tmW, tmY, p);
+    else
+        ptq::ptq_gemm_dequant_kernel<false><<<grid, ptq::kGemmThreads, ptq::kGemmSmemBytes, stream>>>(tmA, h->tmW, tmY, p);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    PTQ_CUDA(cudaGetLastError());
+    return PTQ_OK;
+}
+
+ptq_status_t validate_forward(const ptq_linear *h, const void *x, int B, const void *y)
+{
+    if (!h || !x || !y) return fail(PTQ_ERR_NULL, "handle, x and y must not be NULL");
+    if (B < 1) return fail(PTQ_ERR_SHAPE, "B must be >= 1 (got %d)", B);
+    const long long M = static_cast<long long>(B) * h->T;
+    if (M > 0x7fffff00ll) return fail(PTQ_ERR_SHAPE, "B*T = %lld is too large", M);
+    if (reinterpret_cast<uintptr_t>(x) % 2 || reinterpret_cast<uintptr_t>(y) % 2)
+        return fail(PTQ_ERR_ALIGN, "x and y must be 2-byte aligned");
+    if (ranges_overlap(x, static_cast<size_t>(M) * h->K * 2, y, static_cast<size_t>(M) * h->N * 2))
+        return fail(PTQ_ERR_VALUE, "x and y overlap");
+    return check_device(h);
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *ptq_status_string(ptq_status_t st)
+{
+    switch (st) {
+        case PTQ_OK: return "PTQ_OK";
+        case PTQ_ERR_NULL: return "PTQ_ERR_NULL";
+        case PTQ_ERR_SHAPE: return "PTQ_ERR_SHAPE";
+        case PTQ_ERR_VALUE: return "PTQ_ERR_VALUE";
+        case PTQ_ERR_ALIGN: return "PTQ_ERR_ALIGN";
+        case PTQ_ERR_ARCH: return "PTQ_ERR_ARCH";
+        case PTQ_ERR_CUDA: return "PTQ_ERR_CUDA";
+        case PTQ_ERR_NOMEM: return "PTQ_ERR_NOMEM";
+        case PTQ_ERR_TIMEOUT: return "PTQ_ERR_TIMEOUT";
+    }
+    return "PTQ_ERR_UNKNOWN";
+}
+
+const char *ptq_last_error(void) { return g_err; }
+
+unsigned long long ptq_kernel_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+void ptq_linear_destroy(ptq_linear_t *h)
+{
+    if (!h) return;
+    cudaFree(h->d_w);
+    cudaFree(h->d_dw);
+    cudaFree(h->d_bias);
+    cudaFree(h->d_s);
+    cudaFree(h->d_rs);
+    cudaFree(h->d_dx);
+    cudaFree(h->d_rdx);
+    cudaFree(h->d_status);
+    delete h;
+}
+
+ptq_status_t ptq_linear_create(ptq_linear_t **out, int K, int N, int T, const int8_t *w_q, const float *w_step,
+                               const float *smooth, const float *act_step, const float *bias, unsigned flags)
+{
+    if (!out) return fail(PTQ_ERR_NULL, "out must not be NULL");
+    *out = nullptr;
+    if (!w_q || !w_step || !smooth || !act_step)
+        return fail(PTQ_ERR_NULL, "w_q, w_step, smooth and act_step must not be NULL");
+    if (K < 1 || K > PTQ_MAX_K || N < 1 || N > PTQ_MAX_N || T < 1 || T > PTQ_MAX_T)
+        return fail(PTQ_ERR_SHAPE, "K, N, T out of range (K=%d N=%d T=%d)", K, N, T);
+    if (flags != PTQ_FLAG_NONE) return fail(PTQ_ERR_VALUE, "flags must be PTQ_FLAG_NONE at create");
+
+    // Parameter values (host-only checks come first so that they are testable without a device).
+    const float lo = std::ldexp(1.0f, -30), hi = std::ldexp(1.0f, 30);
+    bool fast = true;
+    for (int k = 0; k < K; ++k) {
+        if (!(smooth[k] > 0.0f) || !std::isfinite(smooth[k]))
+            return fail(PTQ_ERR_VALUE, "smooth[%d] = %g must be finite and > 0", k, smooth[k]);
+        if (smooth[k] < lo || smooth[k] > hi) fast = false;
+    }
+    for (int t = 0; t < T; ++t) {
+        if (!(act_step[t] > 0.0f) || !std::isfinite(act_step[t]))
+            return fail(PTQ_ERR_VALUE, "act_step[%d] = %g must be finite and > 0", t, act_step[t]);
+        if (act_step[t] < lo || act_step[t] > hi) fast = false;
+    }
+    for (int n = 0; n < N; ++n) {
+        if (!(w_step[n] > 0.0f) || !std::isfinite(w_step[n]))
+            return fail(PTQ_ERR_VALUE, "w_step[%d] = %g must be finite and > 0", n, w_step[n]);
+        if (bias && !std::isfinite(bias[n])) return fail(PTQ_ERR_VALUE, "bias[%d] is not finite", n);
+    }
+    for (long long i = 0; i < static_cast<long long>(N) * K; ++i)
+        if (w_q[i] == -128)
+            return fail(PTQ_ERR_VALUE, "w_q[%lld] = -128 is outside the symmetric range [-127,127]", i);
+
+    int dev = -1;
+    PTQ_CUDA(cudaGetDevice(&dev));
+    cudaDeviceProp prop;
+    PTQ_CUDA(cudaGetDeviceProperties(&prop, dev));
+    if (prop.major != 10 || prop.minor != 0)
+        return fail(PTQ_ERR_ARCH, "device %d is compute capability %d.%d; this library needs 10.0 (sm_100a)", dev,
+                    prop.major, prop.minor);
+
+    ptq_linear *h = new (std::nothrow) ptq_linear();
+    if (!h) return fail(PTQ_ERR_NOMEM, "host allocation failed");
+    h->K = K;
+    h->N = N;
+    h->T = T;
+    h->Kpad = round_up(K, 16);
+    h->device = dev;
+    h->num_sms = prop.multiProcessorCount;
+    h->fast_div = fast;
+    h->n_tiles = (N + ptq::kMaxBN - 1) / ptq::kMaxBN;
+    if (h->n_tiles == 1)
+        h->BN = round_up(N, 16);
+    else
+        h->BN = round_up((N + h->n_tiles - 1) / h->n_tiles, 64);
+    h->k_blocks = (K + ptq::kBK - 1) / ptq::kBK;
+    h->last_mmas = (K - (h->k_blocks - 1) * ptq::kBK + 31) / 32;
+
+    const int Npad = h->n_tiles * h->BN;
+    const int Nvec = round_up(Npad, 64) + 64;
+    const int Kvec = round_up(K, 16);
+    std::vector<int8_t> wpad(static_cast<size_t>(Npad) * h->Kpad, 0);
+    for (int n = 0; n < N; ++n) std::memcpy(&wpad[static_cast<size_t>(n) * h->Kpad], w_q + static_cast<size_t>(n) * K, K);
+    std::vector<float> rs(Kvec, 1.0f), sp(Kvec, 1.0f), rdx(T);
+    for (int k = 0; k < K; ++k) {
+        sp[k] = smooth[k];
+        rs[k] = 1.0f / smooth[k];
+    }
+    for (int t = 0; t < T; ++t) rdx[t] = 1.0f / act_step[t];
+
+    ptq_status_t st = PTQ_OK;
+    do {
+        if ((st = upload(reinterpret_cast<void **>(&h->d_w), wpad.data(), wpad.size(), wpad.size())) != PTQ_OK) break;
+        if ((st = upload(reinterpret_cast<void **>(&h->d_dw), w_step, sizeof(float) * N, sizeof(float) * Nvec)) != PTQ_OK) break;
+        if ((st = upload(reinterpret_cast<void **>(&h->d_bias), bias, bias ? sizeof(float) * N : 0, sizeof(float) * Nvec)) != PTQ_OK) break;
+        if ((st = upload(reinterpret_cast<void **>(&h->d_s), sp.data(), sizeof(float) * Kvec, sizeof(float) * Kvec)) != PTQ_OK) break;
+        if ((st = upload(reinterpret_cast<void **>(&h->d_rs), rs.data(), sizeof(float) * Kvec, sizeof(float) * Kvec)) != PTQ_OK) break;
+        if ((st = upload(reinterpret_cast<void **>(&h->d_dx), act_step, sizeof(float) * T, sizeof(float) * T)) != PTQ_OK) break;
+        if ((st = upload(reinterpret_cast<void **>(&h->d_rdx), rdx.data(), sizeof(float) * T, sizeof(float) * T)) != PTQ_OK) break;
+        if ((st = upload(reinterpret_cast<void **>(&h->d_status), nullptr, 0, sizeof(unsigned))) != PTQ_OK) break;
+        st = make_map_2d(&h->tmW, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, h->d_w, static_cast<unsigned long long>(K),
+                         static_cast<unsigned long long>(Npad), static_cast<unsigned long long>(h->Kpad), ptq::kBK,
+                         static_cast<unsigned>(h->BN));
+    } while (0);
+    if (st != PTQ_OK) {
+        char keep[sizeof(g_err)];
+        std::memcpy(keep, g_err, sizeof(keep));
+        ptq_linear_destroy(h);
+        std::memcpy(g_err, keep, sizeof(keep));
+        return st;
+    }
+    *out = h;
+    return PTQ_OK;
+}
+
+size_t ptq_linear_workspace_bytes(const ptq_linear_t *h, int B, unsigned flags)
+{
+    if (!h || B < 1) return 0;
+    if ((flags & PTQ_FLAG_FUSED_PROLOGUE) && ptq_linear_fused_supported(h)) return 0;
+    return static_cast<size_t>(B) * h->T * h->Kpad;
+}
+
+int ptq_linear_fused_supported(const ptq_linear_t *h)
+{
+    (void)h;
+    return 0;
+}
+
+ptq_status_t ptq_quantize(const ptq_linear_t *h, const void *x_fp16, int B, void *q_int8, void *stream)
+{
+    if (!h || !x_fp16 || !q_int8) return fail(PTQ_ERR_NULL, "handle, x and q must not be NULL");
+    if (B < 1) return fail(PTQ_ERR_SHAPE, "B must be >= 1 (got %d)", B);
+    if (reinterpret_cast<uintptr_t>(x_fp16) % 2) return fail(PTQ_ERR_ALIGN, "x must be 2-byte aligned");
+    ptq_status_t st = check_device(h);
+    if (st != PTQ_OK) return st;
+    const long long M = static_cast<long long>(B) * h->T;
+    if (ranges_overlap(x_fp16, static_cast<size_t>(M) * h->K * 2, q_int8, static_cast<size_t>(M) * h->K))
+        return fail(PTQ_ERR_VALUE, "x and q overlap");
+    return launch_quantize(h, x_fp16, M, q_int8, h->K, static_cast<cudaStream_t>(stream));
+}
+
+ptq_status_t ptq_linear_forward_debug(const ptq_linear_t *h, const void *x_fp16, int B, void *y_fp16,
+                                      void *q_int8_out, void *acc_int32_out, void *workspace,
+                                      size_t workspace_bytes, unsigned flags, void *stream)
+{
+    ptq_status_t st = validate_forward(h, x_fp16, B, y_fp16);
+    if (st != PTQ_OK) return st;
+    if (flags & ~PTQ_FLAG_FUSED_PROLOGUE) return fail(PTQ_ERR_VALUE, "unknown flags 0x%x", flags);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const long long M = static_cast<long long>(B) * h->T;
+    const size_t need = static_cast<size_t>(M) * h->Kpad;
+    if (!workspace) return fail(PTQ_ERR_NULL, "workspace must not be NULL for this layer and these flags");
+    if (workspace_bytes < need)
+        return fail(PTQ_ERR_SHAPE, "workspace has %zu bytes, %zu needed", workspace_bytes, need);
+    if (reinterpret_cast<uintptr_t>(workspace) % 16) return fail(PTQ_ERR_ALIGN, "workspace must be 16-byte aligned");
+    if (ranges_overlap(workspace, need, y_fp16, static_cast<size_t>(M) * h->N * 2) ||
+        ranges_overlap(workspace, need, x_fp16, static_cast<size_t>(M) * h->K * 2))
+        return fail(PTQ_ERR_VALUE, "workspace overlaps x or y");
+    if ((st = launch_quantize(h, x_fp16, M, workspace, h->Kpad, s)) != PTQ_OK) return st;
+    if ((st = launch_gemm(h, workspace, M, y_fp16, acc_int32_out, s)) != PTQ_OK) return st;
+    if (q_int8_out)
+        PTQ_CUDA(cudaMemcpy2DAsync(q_int8_out, h->K, workspace, h->Kpad, h->K, static_cast<size_t>(M),
+                                   cudaMemcpyDeviceToDevice, s));
+    return PTQ_OK;
+}
+
+ptq_status_t ptq_linear_forward(const ptq_linear_t *h, const void *x_fp16, int B, void *y_fp16, void *workspace,
+                                size_t workspace_bytes, unsigned flags, void *stream)
+{
+    return ptq_linear_forward_debug(h, x_fp16, B, y_fp16, nullptr, nullptr, workspace, workspace_bytes, flags, stream);
+}
+
+ptq_status_t ptq_linear_device_status(const ptq_linear_t *h)
+{
+    if (!h) return fail(PTQ_ERR_NULL, "handle must not be NULL");
+    ptq_status_t st = check_device(h);
+    if (st != PTQ_OK) return st;
+    unsigned word = 0;
+    PTQ_CUDA(cudaDeviceSynchronize());
+    PTQ_CUDA(cudaMemcpy(&word, h->d_status, sizeof(word), cudaMemcpyDeviceToHost));
+    if (word) {
+        PTQ_CUDA(cudaMemset(h->d_status, 0, sizeof(word)));
+        return fail(PTQ_ERR_TIMEOUT, "a kernel abandoned a bounded wait (status word 0x%x); its output is undefined", word);
+    }
+    return PTQ_OK;
+}
+
+ptq_status_t ptq_calibrate(int K, int N, int T, const void *xcal_fp16, int Bc, const int8_t *w_q,
+                           const float *w_step, float *smooth_out, float *act_step_out, void *stream)
+{
+    if (!xcal_fp16 || !w_q || !w_step || !smooth_out || !act_step_out)
+        return fail(PTQ_ERR_NULL, "calibrate: pointers must not be NULL");
+    if (K < 1 || K > PTQ_MAX_K || N < 1 || N > PTQ_MAX_N || T < 1 || T > PTQ_MAX_T || Bc < 1)
+        return fail(PTQ_ERR_SHAPE, "calibrate: dimensions out of range (K=%d N=%d T=%d Bc=%d)", K, N, T, Bc);
+    if (reinterpret_cast<uintptr_t>(xcal_fp16) % 2) return fail(PTQ_ERR_ALIGN, "xcal must be 2-byte aligned");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int dev = -1, sms = 0;
+    PTQ_CUDA(cudaGetDevice(&dev));
+    PTQ_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    const long long M = static_cast<long long>(Bc) * T;
+
+    unsigned *d_bits = nullptr;   // [K] maxX bits, then [T] mu bits
+    float *d_out = nullptr;       // [K] s, then [T] dx
+    float *d_dw = nullptr;
+    int8_t *d_w = nullptr;
+    ptq_status_t st = PTQ_OK;
+    auto body = [&]() -> ptq_status_t {
+        PTQ_CUDA(cudaMalloc(reinterpret_cast<void **>(&d_bits), sizeof(unsigned) * (K + T)));
+        PTQ_CUDA(cudaMalloc(reinterpret_cast<void **>(&d_out), sizeof(float) * (K + T)));
+        PTQ_CUDA(cudaMalloc(reinterpret_cast<void **>(&d_dw), sizeof(float) * N));
+        PTQ_CUDA(cudaMalloc(reinterpret_cast<void **>(&d_w), static_cast<size_t>(N) * K));
+        PTQ_CUDA(cudaMemsetAsync(d_bits, 0, sizeof(unsigned) * (K + T), s));
+        PTQ_CUDA(cudaMemcpyAsync(d_dw, w_step, sizeof(float) * N, cudaMemcpyHostToDevice, s));
+        PTQ_CUDA(cudaMemcpyAsync(d_w, w_q, static_cast<size_t>(N) * K, cudaMemcpyHostToDevice, s));
+        const __half *x = static_cast<const __half *>(xcal_fp16);
+        long long want = (M + 7) / 8;
+        if (want > sms * 8ll) want = sms * 8ll;
+        const int grid = static_cast<int>(want < 1 ? 1 : want);
+        ptq::ptq_calib_colmax_kernel<<<grid, 256, 0, s>>>(x, M, K, d_bits);
+        ptq::ptq_calib_smooth_kernel<<<(K + 127) / 128, 128, 0, s>>>(d_bits, d_w, d_dw, N, K, d_out);
+        ptq::ptq_calib_rowmax_kernel<<<grid, 256, 0, s>>>(x, M, K, T, d_out, d_bits + K);
+        ptq::ptq_calib_step_kernel<<<(T + 127) / 128, 128, 0, s>>>(d_bits + K, T, d_out + K);
+        g_launches.fetch_add(4, std::memory_order_relaxed);
+        PTQ_CUDA(cudaGetLastError());
+        PTQ_CUDA(cudaMemcpyAsync(smooth_out, d_out, sizeof(float) * K, cudaMemcpyDeviceToHost, s));
+        PTQ_CUDA(cudaMemcpyAsync(act_step_out, d_out + K, sizeof(float) * T, cudaMemcpyDeviceToHost, s));
+        PTQ_CUDA(cudaStreamSynchronize(s));
+        return PTQ_OK;
+    };
+    st = body();
+    cudaFree(d_bits);
+    cudaFree(d_out);
+    cudaFree(d_dw);
+    cudaFree(d_w);
+    return st;
+}
+
+}  // extern "C"

@@ -1,0 +1,329 @@
+// G1 + E1: integer GEMM on the 5th-generation tensor cores with the dequantization fused into
+// the epilogue (Sec. 5.1:  Y = diag(Delta_W) (W-bar X-bar) diag(Delta_X);  Appendix B.1 parts 3-4).
+//
+//   acc[m,n] = sum_k q[m,k] * Wq[n,k]                       tcgen05.mma kind::i8, s32 in TMEM
+//   y[m,n]   = fp16( float(acc) * dx[m mod T] * dw[n] + bias[n] )
+//
+// The rank-1 scaling is applied to the accumulator as it leaves TMEM, so neither the int32
+// product nor an [M,N] step-size tensor ever reaches HBM.
+//
+// One persistent CTA per SM, 6 warps:
+//   warp 0      TMA producer: A tile 128 x 128 B of codes and B tile BN x 128 B of weights per
+//               stage, both written with the 128-byte swizzle, completion on a "full" mbarrier
+//   warp 1      owns TMEM (512 columns = two 128 x 256 accumulators) and issues the MMAs; a
+//               tcgen05.commit frees each shared-memory stage and publishes each accumulator
+//   warps 2..5  epilogue: tcgen05.ld (each warp its own 32-lane quarter), scale, convert, stage the
+//               fp16 tile in swizzled shared memory and write it with a TMA store
+// While the epilogue drains accumulator i the MMA warp already fills accumulator i^1.
+#pragma once
+
+#include <cuda_fp16.h>
+#include <stdint.h>
+
+#include "ptx_sm100.cuh"
+
+namespace ptq {
+
+constexpr int kBM = 128;                                  // rows per tile = TMEM lanes
+constexpr int kBK = 128;                                  // bytes of K per stage row (one swizzle row)
+constexpr int kMaxBN = 256;                               // columns per accumulator
+constexpr int kStages = 4;
+constexpr int kATileBytes = kBM * kBK;                    // 16 KB
+constexpr int kBTileBytes = kMaxBN * kBK;                 // 32 KB
+constexpr int kStageBytes = kATileBytes + kBTileBytes;
+constexpr int kNumEpiWarps = 4;
+constexpr int kStoreBoxCols = 64;                         // fp16 columns per TMA store box (128 B)
+constexpr int kStoreBoxBytes = 32 * kStoreBoxCols * 2;    // 32 rows x 128 B
+constexpr int kStagingBytesPerWarp = 2 * kStoreBoxBytes;  // double buffered
+constexpr int kGemmThreads = 32 * (2 + kNumEpiWarps);
+constexpr int kTmemCols = 512;
+constexpr int kNumBarriers = 2 * kStages + 4;
+constexpr int kGemmSmemBytes =
+    1024 + kStages * kStageBytes + kNumEpiWarps * kStagingBytesPerWarp + kNumBarriers * 8 + 16;
+
+struct GemmParams {
+    long long M;
+    int N, K, T;
+    int BN;            // columns per tile: multiple of 16; multiple of 64 when n_tiles > 1
+    int n_tiles, m_tiles;
+    int k_blocks;      // ceil(K / 128)
+    int last_mmas;     // MMAs (K = 32 each) in the last k-block: ceil((K - 128 (k_blocks-1)) / 32)
+    const float *dx;   // [T]
+    const float *dw;   // [>= n_tiles*BN + 64], zero padded
+    const float *bias; // same length, zeros when the layer has no bias
+    __half *y;         // [M,N]
+    int32_t *acc_out;  // [M,N] or nullptr (parity tap)
+    unsigned *status;  // device status word
+    int use_tma_store; // y is written by TMA (needs N % 8 == 0 and a 16-byte aligned y)
+    int y_vec2;        // plain-store path may use 4-byte stores (N even, y 4-byte aligned)
+};
+
+// --- epilogue helpers -------------------------------------------------------------------------
+
+// y = float(acc) * dx * dw + bias with one rounding per operation (mul, then fma).
+__device__ __forceinline__ float dequant_one(uint32_t acc, float dxr, float dwn, float bn)
+{
+    return __fmaf_rn(__fmul_rn(__int2float_rn(static_cast<int>(acc)), dxr), dwn, bn);
+}
+
+__device__ __forceinline__ uint32_t pack_half2(float a, float b)
+{
+    __half2 h = __floats2half2_rn(a, b);
+    return *reinterpret_cast<uint32_t *>(&h);
+}
+
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint4 v)
+{
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
+                 : "memory");
+}
+
+// Convert 32 accumulator columns of this thread's row and write them as four 16-byte chunks of the
+// row's 128-byte line in the staging buffer (chunk index XOR (row & 7): the 128-byte swizzle the
+// store's tensor map expects, which also spreads the 32 rows over all banks).
+__device__ __forceinline__ void convert_stage32(const uint32_t (&v)[32], int half, float dxr, const float *dw,
+                                                const float *bias, uint32_t row_addr, int lane)
+{
+#pragma unroll
+    for (int jj = 0; jj < 4; ++jj) {
+        const float4 w0 = __ldg(reinterpret_cast<const float4 *>(dw + 8 * jj));
+        const float4 w1 = __ldg(reinterpret_cast<const float4 *>(dw + 8 * jj + 4));
+        const float4 b0 = __ldg(reinterpret_cast<const float4 *>(bias + 8 * jj));
+        const float4 b1 = __ldg(reinterpret_cast<const float4 *>(bias + 8 * jj + 4));
+        uint4 o;
+        o.x = pack_half2(dequant_one(v[8 * jj + 0], dxr, w0.x, b0.x), dequant_one(v[8 * jj + 1], dxr, w0.y, b0.y));
+        o.y = pack_half2(dequant_one(v[8 * jj + 2], dxr, w0.z, b0.z), dequant_one(v[8 * jj + 3], dxr, w0.w, b0.w));
+        o.z = pack_half2(dequant_one(v[8 * jj + 4], dxr, w1.x, b1.x), dequant_one(v[8 * jj + 5], dxr, w1.y, b1.y));
+        o.w = pack_half2(dequant_one(v[8 * jj + 6], dxr, w1.z, b1.z), dequant_one(v[8 * jj + 7], dxr, w1.w, b1.w));
+        const int chunk = half * 4 + jj;
+        st_shared_v4(row_addr + (static_cast<uint32_t>(chunk ^ (lane & 7)) << 4), o);
+    }
+}
+
+// Plain masked stores of 32 columns of this thread's row (any N, any alignment of y).
+__device__ __forceinline__ void convert_store32_plain(const uint32_t (&v)[32], float dxr, const float *dw,
+                                                      const float *bias, __half *yrow, int n_first, int N,
+                                                      bool vec2)
+{
+#pragma unroll
+    for (int i = 0; i < 32; i += 2) {
+        const int n = n_first + i;
+        if (n >= N) break;
+        const float a = dequant_one(v[i], dxr, __ldg(dw + i), __ldg(bias + i));
+        const float b = dequant_one(v[i + 1], dxr, __ldg(dw + i + 1), __ldg(bias + i + 1));
+        if (vec2 && n + 1 < N) {
+            *reinterpret_cast<__half2 *>(yrow + n) = __floats2half2_rn(a, b);
+        } else {
+            yrow[n] = __float2half_rn(a);
+            if (n + 1 < N) yrow[n + 1] = __float2half_rn(b);
+        }
+    }
+}
+
+__device__ __forceinline__ void store_acc32(const uint32_t (&v)[32], int32_t *arow, int n_first, int N)
+{
+#pragma unroll
+    for (int i = 0; i < 32; ++i)
+        if (n_first + i < N) arow[n_first + i] = static_cast<int32_t>(v[i]);
+}
+
+// Epilogue of one 128 x BN accumulator for one warp (its 32-lane quarter).  `tmem_row` addresses the
+// warp's lanes and the accumulator's first column.  Returns the updated count of staged boxes.
+template <bool kDebugAcc>
+__device__ __forceinline__ uint32_t epilogue_tile(const GemmParams &p, const CUtensorMap *tmY, uint32_t tmem_row,
+                                                  long long m_row0, int n0, float dxr, uint32_t staging,
+                                                  uint32_t nboxes, int lane)
+{
+    const long long m = m_row0 + lane;
+    const bool row_ok = m < p.M;
+    for (int c0 = 0; c0 < p.BN; c0 += kStoreBoxCols) {
+        uint32_t v0[32], v1[32];
+        tmem_ld_32x32(tmem_row + c0, v0);
+        tmem_ld_32x32(tmem_row + c0 + 32, v1);
+        tmem_ld_wait();
+        const int n_first = n0 + c0;
+        if (kDebugAcc) {
+            if (p.acc_out != nullptr && row_ok) {
+                store_acc32(v0, p.acc_out + m * p.N, n_first, p.N);
+                store_acc32(v1, p.acc_out + m * p.N, n_first + 32, p.N);
+            }
+        }
+        if (p.use_tma_store) {
+            const uint32_t buf = staging + (nboxes & 1u) * kStoreBoxBytes;
+            if (nboxes >= 2u && lane == 0) bulk_wait_group_read<1>();   // the box that used this buffer was read
+            __syncwarp();
+            const uint32_t row_addr = buf + static_cast<uint32_t>(lane) * 128u;
+            convert_stage32(v0, 0, dxr, p.dw + n_first, p.bias + n_first, row_addr, lane);
+            convert_stage32(v1, 1, dxr, p.dw + n_first + 32, p.bias + n_first + 32, row_addr, lane);
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+                if (n_first < p.N && m_row0 < p.M)
+                    tma_store_2d(tmY, n_first, static_cast<int>(m_row0), buf);   // clipped at N and M
+                bulk_commit_group();
+            }
+            ++nboxes;
+        } else if (row_ok) {
+            __half *yrow = p.y + m * p.N;
+            convert_store32_plain(v0, dxr, p.dw + n_first, p.bias + n_first, yrow, n_first, p.N, p.y_vec2 != 0);
+            convert_store32_plain(v1, dxr, p.dw + n_first + 32, p.bias + n_first + 32, yrow, n_first + 32, p.N,
+                                  p.y_vec2 != 0);
+        }
+    }
+    return nboxes;
+}
+
+// --- the kernel ---------------------------------------------------------------------------------
+
+template <bool kDebugAcc>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+ptq_gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
+                        const __grid_constant__ CUtensorMap tmY, const GemmParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;                    // swizzled tiles need 1024-byte alignment
+    uint8_t *base_ptr = smem_raw + (base - raw);
+    const uint32_t staging_base = base + kStages * kStageBytes;
+    const uint32_t bar_off = kStages * kStageBytes + kNumEpiWarps * kStagingBytesPerWarp;
+    const uint32_t bar_base = base + bar_off;
+    auto full_bar = [&](uint32_t s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](uint32_t s) { return bar_base + 8u * (kStages + s); };
+    auto tfull_bar = [&](uint32_t b) { return bar_base + 8u * (2 * kStages + b); };
+    auto tempty_bar = [&](uint32_t b) { return bar_base + 8u * (2 * kStages + 2 + b); };
+    volatile uint32_t *tmem_holder = reinterpret_cast<volatile uint32_t *>(base_ptr + bar_off + kNumBarriers * 8);
+    volatile uint32_t *abort_flag = tmem_holder + 1;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (uint32_t s = 0; s < kStages; ++s) {
+            mbar_init(full_bar(s), 1);
+            mbar_init(empty_bar(s), 1);
+        }
+        for (uint32_t b = 0; b < 2; ++b) {
+            mbar_init(tfull_bar(b), 1);
+            mbar_init(tempty_bar(b), kNumEpiWarps);
+        }
+        *abort_flag = 0u;
+        fence_mbar_init();
+        prefetch_tensormap(&tmA);
+        prefetch_tensormap(&tmW);
+        if (p.use_tma_store) prefetch_tensormap(&tmY);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(const_cast<uint32_t *>(tmem_holder)), kTmemCols);
+        tmem_relinquish_alloc_permit();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_holder;
+
+    const int total_tiles = p.m_tiles * p.n_tiles;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0, issued = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+                const int m_tile = tile / p.n_tiles;
+                const int n_tile = tile - m_tile * p.n_tiles;
+                for (int kb = 0; kb < p.k_blocks; ++kb) {
+                    if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status)) {
+                        ok = false;
+                        break;
+                    }
+                    const uint32_t a_dst = base + stage * kStageBytes;
+                    mbar_arrive_expect_tx(full_bar(stage), static_cast<uint32_t>(kATileBytes + p.BN * kBK));
+                    tma_load_2d(a_dst, &tmA, kb * kBK, m_tile * kBM, full_bar(stage));
+                    tma_load_2d(a_dst + kATileBytes, &tmW, kb * kBK, n_tile * p.BN, full_bar(stage));
+                    ++issued;
+                    if (++stage == kStages) {
+                        stage = 0;
+                        phase ^= 1u;
+                    }
+                }
+            }
+            if (!ok) {
+                // Error path only: let this thread's own loads land before the CTA gives up its
+                // shared memory (bounded; each stage's last load is at most microseconds away).
+                for (uint32_t s = 0; s < kStages; ++s) {
+                    const uint32_t uses = (issued + kStages - 1u - s) / kStages;
+                    if (uses == 0u) continue;
+                    for (int i = 0; i < 200000 && !mbar_try_wait(full_bar(s), (uses - 1u) & 1u); ++i) {
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = make_idesc_s8(kBM, p.BN);
+            uint32_t stage = 0, phase = 0, buf = 0, bphase = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+                if (!mbar_wait(tempty_bar(buf), bphase ^ 1u, abort_flag, p.status)) break;
+                tc_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + buf * kMaxBN;
+                for (int kb = 0; kb < p.k_blocks; ++kb) {
+                    if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after_sync();
+                    const uint32_t a_addr = base + stage * kStageBytes;
+                    const uint64_t a_desc = make_smem_desc_sw128(a_addr);
+                    const uint64_t b_desc = make_smem_desc_sw128(a_addr + kATileBytes);
+                    const int nmma = (kb == p.k_blocks - 1) ? p.last_mmas : (kBK / 32);
+                    for (int j = 0; j < nmma; ++j)   // 32 bytes of K per MMA: +2 in the (>>4) address field
+                        mma_i8_ss(d_tmem, a_desc + 2u * j, b_desc + 2u * j, idesc, (kb | j) != 0 ? 1u : 0u);
+                    mma_commit(empty_bar(stage));    // the stage is free once these MMAs have read it
+                    if (++stage == kStages) {
+                        stage = 0;
+                        phase ^= 1u;
+                    }
+                }
+                if (!ok) break;
+                mma_commit(tfull_bar(buf));          // accumulator complete
+                buf ^= 1u;
+                if (buf == 0u) bphase ^= 1u;
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue warps
+        const int quarter = warp & 3;                // TMEM lanes [32*quarter, 32*quarter+32)
+        const uint32_t staging = staging_base + static_cast<uint32_t>(warp - 2) * kStagingBytesPerWarp;
+        uint32_t buf = 0, bphase = 0, nboxes = 0;
+        for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+            const int m_tile = tile / p.n_tiles;
+            const int n_tile = tile - m_tile * p.n_tiles;
+            const long long m_row0 = static_cast<long long>(m_tile) * kBM + quarter * 32;
+            const long long m = m_row0 + lane;
+            const float dxr = (m < p.M) ? __ldg(p.dx + static_cast<int>(m % p.T)) : 0.0f;
+            bool got = mbar_wait(tfull_bar(buf), bphase, abort_flag, p.status);
+            got = __all_sync(0xffffffffu, got);
+            if (!got) break;
+            tc_fence_after_sync();
+            const uint32_t tmem_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * kMaxBN;
+            nboxes = epilogue_tile<kDebugAcc>(p, &tmY, tmem_row, m_row0, n_tile * p.BN, dxr, staging, nboxes, lane);
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty_bar(buf));
+            buf ^= 1u;
+            if (buf == 0u) bphase ^= 1u;
+        }
+        if (lane == 0) bulk_wait_group<0>();         // all of this thread's stores have completed
+    }
+
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+}  // namespace ptq
