@@ -1,0 +1,200 @@
+"""GPU parity tests: the CUDA path, called through the C ABI, against the CPU oracle on the same
+seeded inputs.  int8 codes and int32 accumulators must match bit for bit; fp16 outputs within
+max(2^-10 |ref|, 1e-3)."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2412_20386_b200 import workloads as wl
+from parity_util import assert_y_close, check_layer, layer_inputs
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def env():
+    import torch
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    import __graft_entry__ as entry
+    entry.build()
+    import paper_2412_20386_b200 as ptq
+    ptq.load_library()          # raises if the CUDA library is missing: there is no fallback
+    torch.cuda.set_device(0)
+    return ptq, torch
+
+
+CFG = wl.configs()
+
+
+def test_config0_vim_ti_out_proj_single_image(env):
+    ptq, torch = env
+    check_layer(ptq, torch, CFG[0][0])
+
+
+@pytest.mark.parametrize("idx", [0, 1, 2, 3, 4 * 23 + 0, 4 * 11 + 1, 4 * 7 + 2, 4 * 17 + 3])
+def test_config1_vim_ti_block_linears_batch64(env, idx):
+    ptq, torch = env
+    clip = check_layer(ptq, torch, CFG[1][idx], full=True)
+    assert clip > 0      # heavy tails beyond the calibration range do clip
+
+
+@pytest.mark.parametrize("idx", [0, 1])
+def test_config2_vim_s_batch128(env, idx):
+    ptq, torch = env
+    check_layer(ptq, torch, CFG[2][idx], full=False)
+
+
+@pytest.mark.parametrize("idx", [0, 1])
+def test_config3_vim_b_batch256(env, idx):
+    ptq, torch = env
+    check_layer(ptq, torch, CFG[3][idx], full=False)
+
+
+@pytest.mark.parametrize("idx", range(8))
+def test_config4_vmamba_stages_batch64(env, idx):
+    ptq, torch = env
+    check_layer(ptq, torch, CFG[4][idx], full=False)
+
+
+def test_quantizer_all_fp16_inputs_many_scales(env):
+    # every binary16 bit pattern against 8 token steps x 64 channel scales (vector kernel), and against
+    # 5 x 12 (scalar kernel); this is also the check of the reciprocal + FMA division route.
+    ptq, torch = env
+    rng = np.random.default_rng(11)
+    for (T, K) in ((8, 64), (5, 12)):
+        s = np.exp(rng.uniform(np.log(2e-3), np.log(3e2), K)).astype(np.float32)
+        dx = np.exp(rng.uniform(np.log(1e-3), np.log(1e1), T)).astype(np.float32)
+        s[0], dx[0] = 1.0, 1.0
+        s[1], dx[1] = 3.0, 1.0 / 3.0
+        B = 65536
+        M = B * T
+        base = (np.arange(M, dtype=np.int64) // T).astype(np.uint16)              # image b carries pattern b
+        x = np.repeat(base[:, None], K, axis=1)
+        x = (x + (np.arange(K, dtype=np.uint16) * 977)[None, :]).astype(np.uint16)   # every channel sees all patterns
+        xh = x.view(np.float16).reshape(B, T, K)
+        wq = np.ones((4, K), np.int8)
+        layer = ptq.PtqLinear(wq, np.ones(4, np.float32), s, dx)
+        q = layer.quantize(torch.from_numpy(xh).cuda()).cpu().numpy().reshape(M, K)
+        want = oracle.quantize(xh.reshape(M, K), T, s, dx)
+        assert np.array_equal(q, want)
+
+
+def test_quantizer_scales_outside_reciprocal_range_use_ieee_division(env):
+    ptq, torch = env
+    rng = np.random.default_rng(12)
+    T, K, B = 3, 32, 700
+    s = np.exp(rng.uniform(-2, 2, K)).astype(np.float32)
+    dx = np.exp(rng.uniform(-2, 2, T)).astype(np.float32)
+    s[5] = 1e-12
+    s[6] = 3e13
+    dx[1] = 2e-11
+    x = (rng.standard_normal((B, T, K)) * 10.0 ** rng.uniform(-7, 4, (B, T, K))).astype(np.float16)
+    layer = ptq.PtqLinear(np.ones((4, K), np.int8), np.ones(4, np.float32), s, dx)
+    q = layer.quantize(torch.from_numpy(x).cuda()).cpu().numpy().reshape(-1, K)
+    assert np.array_equal(q, oracle.quantize(x.reshape(-1, K), T, s, dx))
+
+
+def test_closed_form_integer_inputs_on_gpu(env):
+    # s = dx = dw = 1 and integer-valued activations: codes equal the inputs and the output is the
+    # exact integer matmul rounded to fp16 (checked against numpy int64, not against the oracle).
+    ptq, torch = env
+    rng = np.random.default_rng(13)
+    B, T, K, N = 5, 61, 160, 72
+    xi = rng.integers(-128, 128, (B, T, K))
+    wq = rng.integers(-2, 3, (N, K)).astype(np.int8)
+    one = lambda n: np.ones(n, np.float32)
+    layer = ptq.PtqLinear(wq, one(N), one(K), one(T))
+    y, q, acc = layer.forward_debug(torch.from_numpy(xi.astype(np.float16)).cuda())
+    exact = xi.reshape(-1, K) @ wq.astype(np.int64).T
+    assert np.array_equal(q.cpu().numpy().reshape(-1, K).astype(np.int64), xi.reshape(-1, K))
+    assert np.array_equal(acc.cpu().numpy().reshape(-1, N).astype(np.int64), exact)
+    assert np.array_equal(y.cpu().numpy().reshape(-1, N).view(np.uint16),
+                          exact.astype(np.float64).astype(np.float16).view(np.uint16))
+
+
+@pytest.mark.parametrize("K,N,T,B", [(12, 384, 197, 2), (384, 44, 197, 3), (96, 8, 7, 40), (1536, 768, 49, 6),
+                                     (40, 300, 3, 50), (8192, 16, 2, 70), (129, 257, 5, 30), (16, 1000, 1, 131)])
+def test_odd_shapes_and_ragged_tiles(env, K, N, T, B):
+    ptq, torch = env
+    spec = wl.LinearSpec(9, K % 97, N % 5, "odd", B, T, K, N, bias=(N % 2 == 0))
+    check_layer(ptq, torch, spec, full=True)
+
+
+def test_unaligned_pointers_take_the_generic_paths(env):
+    ptq, torch = env
+    spec = CFG[0][0]
+    x, wq, dw, bias, s, dx = layer_inputs(spec, B=2)
+    M = 2 * spec.T
+    layer = ptq.PtqLinear(wq, dw, s, dx, bias)
+    xbuf = torch.zeros(x.size + 8, dtype=torch.float16, device="cuda")
+    ybuf = torch.zeros(M * spec.N + 8, dtype=torch.float16, device="cuda")
+    xv = xbuf[1:1 + x.size].view(2, spec.T, spec.K)          # 2-byte aligned only
+    yv = ybuf[1:1 + M * spec.N].view(2, spec.T, spec.N)
+    xv.copy_(torch.from_numpy(x).cuda())
+    layer.forward(xv, y=yv)
+    torch.cuda.synchronize()
+    layer.device_status()
+    y_ref = oracle.linear_forward(x.reshape(M, spec.K), spec.T, wq, dw, s, dx, bias)
+    assert_y_close(yv.cpu().numpy().reshape(M, spec.N), y_ref, "unaligned")
+    assert float(ybuf[0]) == 0.0 and float(ybuf[-7:].abs().max()) == 0.0     # nothing written outside y
+
+
+def test_repeated_runs_are_bit_identical_and_stay_inside_y(env):
+    ptq, torch = env
+    spec = CFG[1][3]
+    x, wq, dw, bias, s, dx = layer_inputs(spec, B=16)
+    layer = ptq.PtqLinear(wq, dw, s, dx, bias)
+    xd = torch.from_numpy(x).cuda()
+    M = 16 * spec.T
+    guard = 4096
+    ybuf = torch.full((M * spec.N + 2 * guard,), -7.0, dtype=torch.float16, device="cuda")
+    yv = ybuf[guard:guard + M * spec.N].view(16, spec.T, spec.N)
+    ws = torch.empty(layer.workspace_bytes(16) + 2 * guard, dtype=torch.uint8, device="cuda")
+    first = None
+    for _ in range(10):
+        layer.forward(xd, y=yv, workspace=ws[guard:guard + layer.workspace_bytes(16)])
+        cur = yv.clone()
+        first = cur if first is None else first
+        assert torch.equal(cur, first)
+    layer.device_status()
+    assert bool((ybuf[:guard] == -7.0).all()) and bool((ybuf[-guard:] == -7.0).all())
+
+
+def test_calibration_kernels_match_oracle_bit_for_bit(env):
+    ptq, torch = env
+    for spec in (CFG[0][0], CFG[1][2], CFG[4][7], CFG[4][0].with_batch(2)):
+        xcal = wl.activations(spec, wl.ROLE_CALIB, B=min(8, spec.B))
+        wq, dw, _ = wl.weights(spec)
+        s, dx = ptq.calibrate(torch.from_numpy(xcal).cuda(), wq, dw)
+        s_ref, dx_ref = oracle.calibrate(xcal, wq, dw)
+        assert np.array_equal(s.view(np.uint32), s_ref.view(np.uint32))
+        assert np.array_equal(dx.view(np.uint32), dx_ref.view(np.uint32))
+    # degenerate: dead channels and positions
+    xcal = np.zeros((2, 3, 16), np.float16)
+    xcal[:, 1, 2] = 3.0
+    wq = np.zeros((4, 16), np.int8)
+    wq[:, 2] = [10, -20, 5, 40]
+    dw = np.array([0.01, 0.01, 0.02, 0.02], np.float32)
+    s, dx = ptq.calibrate(torch.from_numpy(xcal).cuda(), wq, dw)
+    s_ref, dx_ref = oracle.calibrate(xcal, wq, dw)
+    assert np.array_equal(s, s_ref) and np.array_equal(dx, dx_ref)
+
+
+def test_forward_argument_errors_return_codes(env):
+    ptq, torch = env
+    spec = CFG[0][0]
+    x, wq, dw, bias, s, dx = layer_inputs(spec, B=1)
+    layer = ptq.PtqLinear(wq, dw, s, dx, bias)
+    xd = torch.from_numpy(x).cuda()
+    small = torch.empty(16, dtype=torch.uint8, device="cuda")
+    with pytest.raises(ptq.PtqError) as e:
+        layer.forward(xd, workspace=small)
+    assert e.value.status == 2
+    with pytest.raises(ptq.PtqError) as e:
+        layer.forward(xd, flags=64)
+    assert e.value.status == 3
+    y = layer.forward(xd)          # the handle still works after refused calls
+    torch.cuda.synchronize()
+    layer.device_status()
+    assert_y_close(y.cpu().numpy().reshape(-1, spec.N),
+                   oracle.linear_forward(x.reshape(-1, spec.K), spec.T, wq, dw, s, dx, bias), "after errors")
