@@ -1,0 +1,425 @@
+#!/usr/bin/env python
+"""Benchmark of the PTS W8A8 linear path (quantize + integer GEMM + dequantize) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c3] [--impl ours|reference]
+
+One step = one forward pass of every linear layer of the workload configuration over one batch of
+seeded synthetic activations, through the C ABI (`ptq_linear_forward`).  Prints ONE JSON line.
+
+  value          INT8 TOPS = sum_layers 2 M K N / step time, inputs resident in HBM, CUDA events
+  e2e            the same metric with pinned HOST buffers: host->device copy of x, forward,
+                 device->host copy of y, all inside the timed region
+  roofline       the dominant kernel (largest share of the step), timed alone with CUDA events on
+                 the launching stream in the same process; plus `kernels` with every kernel's figure
+  cpu_baseline   the CPU oracle, as it stands, on a bounded row sample of the same workload
+
+With N > 1 (torchrun) every rank runs an independent replica on its own GPU (the path has no
+exchange step: rows are independent and the parameters are replicated), so scaling is weak.
+`--impl reference` times the CPU oracle instead (rank 0 only).
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "PTS W8A8 linear INT8 TOPS (quant+GEMM+dequant)"
+UNIT = "TOPS"
+INT8_OVER_BF16 = 2.0          # nominal dense ratio 4.5 / 2.25 PFLOP/s
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return d, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def layer_ops(spec, B):
+    return 2.0 * B * spec.T * spec.K * spec.N
+
+
+def workload_specs(name):
+    from paper_2412_20386_b200 import workloads as wl
+    idx = int(name[1:])
+    return wl.configs()[idx]
+
+
+# ------------------------------------------------------------------------------------------------
+# clocks
+# ------------------------------------------------------------------------------------------------
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.proc = None
+        self.lines = []
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in self.lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                smax.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(smax) if smax else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle arm (also the cpu_baseline leg of the GPU arm)
+# ------------------------------------------------------------------------------------------------
+def oracle_layer_inputs(spec, rows):
+    """Inputs of one layer restricted to the first `rows` token rows (whole images)."""
+    import oracle
+    from paper_2412_20386_b200 import workloads as wl
+    images = max(1, min(spec.B, (rows + spec.T - 1) // spec.T))
+    x = wl.activations(spec, wl.ROLE_EVAL, B=images).reshape(-1, spec.K)
+    wq, dw, bias = wl.weights(spec)
+    s, dx = oracle.calibrate(wl.activations(spec, wl.ROLE_CALIB), wq, dw)
+    return x, wq, dw, bias, s, dx
+
+
+def time_oracle(specs, target_seconds, repeats=1):
+    """Times the oracle's whole path on the leading rows of every layer; the row count is sized by a
+    short probe so that one pass takes about `target_seconds`.  Returns (TOPS, sample text, seconds)."""
+    import oracle
+    total_ops_full = sum(layer_ops(sp, sp.B) for sp in specs)
+    plans = []
+    for sp in specs:
+        probe_rows = min(sp.M, 256)
+        x, wq, dw, bias, s, dx = oracle_layer_inputs(sp, probe_rows)
+        t0 = time.perf_counter()
+        oracle.linear_forward(x, sp.T, wq, dw, s, dx, bias, rows=(0, probe_rows))
+        dt = max(time.perf_counter() - t0, 1e-6)
+        share = layer_ops(sp, sp.B) / total_ops_full
+        rows = int(min(sp.M, max(probe_rows, probe_rows * (target_seconds * share) / dt)))
+        plans.append((sp, rows))
+    ops = 0.0
+    secs = 0.0
+    data = [(sp, rows, oracle_layer_inputs(sp, rows)) for sp, rows in plans]
+    for _ in range(repeats):
+        for sp, rows, (x, wq, dw, bias, s, dx) in data:
+            rows = min(rows, x.shape[0])
+            t0 = time.perf_counter()
+            oracle.linear_forward(x, sp.T, wq, dw, s, dx, bias, rows=(0, rows))
+            secs += time.perf_counter() - t0
+            ops += 2.0 * rows * sp.K * sp.N
+    sample = "; ".join("%s L%d %s: first %d of %d rows" % ("c%d" % sp.config, sp.layer, sp.name, rows, sp.M)
+                       for sp, rows in plans[:6])
+    if len(plans) > 6:
+        sample += "; ... (%d layers)" % len(plans)
+    return ops / secs / 1e12, sample, secs
+
+
+def run_reference(args, specs, rank):
+    if rank != 0:
+        return
+    import oracle
+    per_step = 2.0
+    t_all = time.perf_counter()
+    for _ in range(args.warmup):
+        time_oracle(specs, per_step * 0.25)
+    vals = []
+    sample = ""
+    for _ in range(args.steps):
+        v, sample, _ = time_oracle(specs, per_step)
+        vals.append(v)
+    # whole-run throughput = total ops / total time = harmonic-style mean over equal-length steps
+    value = len(vals) / sum(1.0 / v for v in vals)
+    cores = oracle.num_threads()
+    out = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": 1e3 * (time.perf_counter() - t_all) / max(1, args.steps + args.warmup),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+        "config": {"workload": args.workload, "layers": len(specs)},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(out))
+
+
+# ------------------------------------------------------------------------------------------------
+# GPU arm
+# ------------------------------------------------------------------------------------------------
+def event_times_ms(torch, fn, iters):
+    """Average device time of fn() per call, each call bracketed by its own CUDA events on the
+    current stream (the stream the library launches on)."""
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(iters)]
+    torch.cuda.synchronize()
+    for a, b in evs:
+        a.record()
+        fn()
+        b.record()
+    torch.cuda.synchronize()
+    ts = [a.elapsed_time(b) for a, b in evs]
+    return sum(ts) / len(ts), min(ts), statistics.median(ts)
+
+
+def run_ours(args, specs, rank, world, local_rank):
+    import torch
+    import __graft_entry__ as entry
+    if rank == 0:
+        entry.build()
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+    import paper_2412_20386_b200 as ptq
+    from paper_2412_20386_b200 import workloads as wl
+    L = ptq.load_library()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    peaks, peaks_kind = load_peaks()
+
+    flags = ptq.FLAG_FUSED_PROLOGUE if args.path == "fused" else 0
+    layers = []
+    for sp in specs:
+        x_host = torch.from_numpy(wl.activations(sp, wl.ROLE_EVAL)).pin_memory()
+        wq, dw, bias = wl.weights(sp)
+        xcal = torch.from_numpy(wl.activations(sp, wl.ROLE_CALIB)).to(dev)
+        s, dx = ptq.calibrate(xcal, wq, dw)                      # Q0 on the GPU
+        layer = ptq.PtqLinear(wq, dw, s, dx, bias)
+        x_dev = x_host.to(dev)
+        y_dev = torch.empty((sp.B, sp.T, sp.N), dtype=torch.float16, device=dev)
+        y_host = torch.empty((sp.B, sp.T, sp.N), dtype=torch.float16).pin_memory()
+        ws_bytes = layer.workspace_bytes(sp.B, flags)
+        ws = torch.empty(max(ws_bytes, 16), dtype=torch.uint8, device=dev)
+        layers.append(dict(spec=sp, layer=layer, x_host=x_host, x=x_dev, y=y_dev, y_host=y_host, ws=ws,
+                           fused=bool(flags and layer.fused_supported())))
+    step_ops = sum(layer_ops(d["spec"], d["spec"].B) for d in layers)
+    touched = sum(d["x"].numel() * 2 + d["y"].numel() * 2 for d in layers)
+
+    def step():
+        for d in layers:
+            d["layer"].forward(d["x"], y=d["y"], workspace=d["ws"], flags=flags)
+
+    def step_e2e():
+        for d in layers:
+            d["x"].copy_(d["x_host"], non_blocking=True)
+            d["layer"].forward(d["x"], y=d["y"], workspace=d["ws"], flags=flags)
+            d["y_host"].copy_(d["y"], non_blocking=True)
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing -------------------------------------------------------------
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    n0 = ptq.binding.kernel_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier()
+    launches = ptq.binding.kernel_launch_count() - n0
+    ms_total = e0.elapsed_time(e1)
+    clocks = sampler.stop()
+    for d in layers:
+        d["layer"].device_status()
+
+    # ---- end to end with host buffers -------------------------------------------------------
+    for _ in range(min(args.warmup, 3)):
+        step_e2e()
+    barrier()
+    e2e_steps = max(3, min(args.steps, 20))
+    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    f0.record()
+    for _ in range(e2e_steps):
+        step_e2e()
+    f1.record()
+    barrier()
+    ms_e2e = f0.elapsed_time(f1) / e2e_steps
+
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total, ms_e2e = float(t[0]), float(t[1])
+    ms_step = ms_total / args.steps
+    value = world * step_ops / (ms_step * 1e-3) / 1e12
+    e2e_value = world * step_ops / (ms_e2e * 1e-3) / 1e12
+
+    if rank != 0:
+        return
+
+    # ---- per-kernel timing (rank 0): each kernel alone, events around every launch ----------
+    int8_peak = peaks["bf16_tflops_sustained"] * INT8_OVER_BF16
+    hbm_peak = peaks["hbm_gbs"]
+    kernels = []
+    iters = max(10, min(args.steps, 50))
+    for d in layers:
+        sp, layer = d["spec"], d["layer"]
+        M, K, N = sp.M, sp.K, sp.N
+        tag = "c%d.L%d.%s" % (sp.config, sp.layer, sp.name)
+        if d["fused"]:
+            avg, mn, med = event_times_ms(torch, lambda: layer.forward(d["x"], y=d["y"], workspace=d["ws"], flags=flags), iters)
+            byts = 2.0 * M * K + N * K + 2.0 * M * N
+            kernels.append(dict(kernel="ptq_fused_linear_kernel", layer=tag, ms=avg, ms_min=mn, ops=2.0 * M * K * N, bytes=byts))
+        else:
+            pitch = layer.code_pitch()
+            codes = d["ws"][:M * pitch]
+            qdense = torch.empty((sp.B, sp.T, K), dtype=torch.int8, device=dev)
+            avg, mn, med = event_times_ms(torch, lambda: layer.quantize(d["x"], q=qdense), iters)
+            kernels.append(dict(kernel="ptq_quantize_kernel", layer=tag, ms=avg, ms_min=mn, ops=0.0, bytes=3.0 * M * K))
+            layer.forward(d["x"], y=d["y"], workspace=d["ws"], flags=0)      # leaves valid codes in ws
+            avg, mn, med = event_times_ms(torch, lambda: layer.gemm_dequant(codes, sp.B, y=d["y"]), iters)
+            kernels.append(dict(kernel="ptq_gemm_dequant_kernel", layer=tag, ms=avg, ms_min=mn, ops=2.0 * M * K * N,
+                                bytes=1.0 * M * K + N * K + 2.0 * M * N))
+            del qdense
+    for k in kernels:
+        t = k["ms"] * 1e-3
+        k["tops"] = k["ops"] / t / 1e12
+        k["gbs"] = k["bytes"] / t / 1e9
+        k["frac_tensor"] = k["tops"] / int8_peak
+        k["frac_hbm"] = k["gbs"] / hbm_peak
+        k["bound"] = "tensor" if k["frac_tensor"] >= k["frac_hbm"] else "hbm"
+    # the dominant kernel is the one with the largest share of the step when timed alone
+    agg = {}
+    for k in kernels:
+        agg.setdefault(k["kernel"], 0.0)
+        agg[k["kernel"]] += k["ms"]
+    dom_name = max(agg, key=agg.get)
+    dom = max((k for k in kernels if k["kernel"] == dom_name), key=lambda k: k["ms"])
+    if dom["bound"] == "tensor":
+        roof = {"bound": "tensor", "achieved": dom["tops"], "peak": int8_peak, "unit": "TFLOP/s",
+                "frac": dom["frac_tensor"]}
+    else:
+        roof = {"bound": "hbm", "achieved": dom["gbs"], "peak": hbm_peak, "unit": "GB/s", "frac": dom["frac_hbm"]}
+    roof.update({"kernel": dom["kernel"], "layer": dom["layer"], "ms_per_launch": dom["ms"],
+                 "peak_source": "%s (%s)" % (("2 x bf16_tflops_sustained" if dom["bound"] == "tensor" else "hbm_gbs"),
+                                             peaks_kind),
+                 "traffic": TRAFFIC.get((dom["kernel"], args.workload, dom["layer"].split(".")[-1]))})
+
+    # ---- CPU oracle baseline on a bounded sample -------------------------------------------
+    import oracle
+    cpu_val, cpu_sample, cpu_secs = time_oracle(specs, args.cpu_seconds)
+    cpu = {"value": cpu_val, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+           "sample": cpu_sample, "seconds": cpu_secs}
+
+    h2d = sum(d["x"].numel() * 2 for d in layers)
+    d2h = sum(d["y"].numel() * 2 for d in layers)
+    sp0 = specs[0]
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "int8", "data": "synthetic",
+        "config": {"workload": args.workload, "layers": ["%s %dx%d->%d" % (sp.name, sp.M, sp.K, sp.N) for sp in specs][:8],
+                   "n_layers": len(specs), "batch": sp0.B, "tokens": sp0.T, "path": args.path,
+                   "fused_layers": sum(1 for d in layers if d["fused"]),
+                   "l2": "inputs_larger_than_l2 (%.0f MB touched per step)" % (touched / 1e6)
+                   if touched > 2 * 126e6 else "working set %.0f MB fits L2: L2-warm timing" % (touched / 1e6),
+                   "parallelism": "replicas x%d" % world},
+        "pct_of_int8_peak": {"nominal_4500": 100.0 * value / world / 4500.0,
+                             "measured_2x_bf16_sustained": 100.0 * value / world / int8_peak},
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": ms_e2e},
+        "gpu_launches": int(launches),
+        "roofline": roof,
+        "kernels": [{k2: (round(v, 5) if isinstance(v, float) else v) for k2, v in k.items()} for k in kernels[:16]],
+        "cpu_baseline": cpu,
+    }
+    print(json.dumps(out))
+
+
+# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) from ncu captures of the
+# current kernels; keyed by (kernel, workload, layer).  Empty until a capture of the current code exists.
+TRAFFIC = {}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c3", choices=["c0", "c1", "c2", "c3", "c4"])
+    ap.add_argument("--path", default="unfused", choices=["unfused", "fused"])
+    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    specs = workload_specs(args.workload)
+
+    if args.impl == "reference":
+        run_reference(args, specs, rank)
+        return
+
+    if world > 1:
+        import torch
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        torch.cuda.set_device(local_rank)
+        dist.init_process_group("nccl")
+    try:
+        run_ours(args, specs, rank, world, local_rank)
+    finally:
+        if world > 1:
+            import torch.distributed as dist
+            dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

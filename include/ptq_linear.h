@@ -119,6 +119,19 @@ ptq_status_t ptq_quantize(const ptq_linear_t *h, const void *x_fp16, int B,
                           void *q_int8, void *stream);
 
 /*
+ * G1 + E1 alone (Sec. 5.1; Appendix B.1, parts 3-4): integer GEMM and dequantization on codes that
+ * are already in device memory.
+ *   q_int8     device, [B*T, pitch] int8 codes with pitch = ptq_linear_code_pitch(h) bytes per row
+ *              (K rounded up to 16; bytes beyond K in a row are ignored), 16-byte aligned
+ *   y_fp16     device, [B,T,N] binary16
+ */
+ptq_status_t ptq_linear_gemm_dequant(const ptq_linear_t *h, const void *q_int8, int B, void *y_fp16,
+                                     void *stream);
+
+/* Bytes per row of the code matrix that ptq_linear_gemm_dequant reads and the workspace holds. */
+int ptq_linear_code_pitch(const ptq_linear_t *h);
+
+/*
  * Forward pass with parity taps.  Same as ptq_linear_forward, and additionally writes
  *   q_int8_out     device, [B,T,K] dense int8 codes of Q1, or NULL
  *                  (with PTQ_FLAG_FUSED_PROLOGUE the codes never exist in memory; they are then

@@ -60,6 +60,10 @@ def load_library() -> ctypes.CDLL:
     L.ptq_linear_fused_supported.argtypes = [vp]
     L.ptq_quantize.restype = ci
     L.ptq_quantize.argtypes = [vp, vp, ci, vp, vp]
+    L.ptq_linear_gemm_dequant.restype = ci
+    L.ptq_linear_gemm_dequant.argtypes = [vp, vp, ci, vp, vp]
+    L.ptq_linear_code_pitch.restype = ci
+    L.ptq_linear_code_pitch.argtypes = [vp]
     L.ptq_linear_forward_debug.restype = ci
     L.ptq_linear_forward_debug.argtypes = [vp, vp, ci, vp, vp, vp, vp, sz, cu, vp]
     L.ptq_calibrate.restype = ci
@@ -178,6 +182,21 @@ class PtqLinear:
             q = torch.empty((B, self.T, self.K), dtype=torch.int8, device=x.device)
         _check(self._L.ptq_quantize(self._h, x.data_ptr(), B, q.data_ptr(), _stream_ptr(stream)))
         return q
+
+    def code_pitch(self) -> int:
+        return int(self._L.ptq_linear_code_pitch(self._h))
+
+    def gemm_dequant(self, q, B: int, y=None, stream=None):
+        """``ptq_linear_gemm_dequant``: int8 codes [B*T, code_pitch()] -> y fp16 [B,T,N]."""
+        import torch
+        if q.dtype not in (torch.int8, torch.uint8) or not q.is_cuda or not q.is_contiguous():
+            raise ValueError("q must be a contiguous CUDA int8 tensor")
+        if q.numel() < B * self.T * self.code_pitch():
+            raise ValueError("q holds fewer than B*T rows of code_pitch() bytes")
+        if y is None:
+            y = torch.empty((B, self.T, self.N), dtype=torch.float16, device=q.device)
+        _check(self._L.ptq_linear_gemm_dequant(self._h, q.data_ptr(), int(B), y.data_ptr(), _stream_ptr(stream)))
+        return y
 
     def forward_debug(self, x, flags: int = 0, want_q=True, want_acc=True, stream=None):
         """``ptq_linear_forward_debug``: returns (y, q or None, acc or None)."""

@@ -415,6 +415,22 @@ ptq_status_t ptq_quantize(const ptq_linear_t *h, const void *x_fp16, int B, void
     return launch_quantize(h, x_fp16, M, q_int8, h->K, static_cast<cudaStream_t>(stream));
 }
 
+int ptq_linear_code_pitch(const ptq_linear_t *h) { return h ? h->Kpad : 0; }
+
+ptq_status_t ptq_linear_gemm_dequant(const ptq_linear_t *h, const void *q_int8, int B, void *y_fp16, void *stream)
+{
+    if (!h || !q_int8 || !y_fp16) return fail(PTQ_ERR_NULL, "handle, q and y must not be NULL");
+    if (B < 1) return fail(PTQ_ERR_SHAPE, "B must be >= 1 (got %d)", B);
+    if (reinterpret_cast<uintptr_t>(q_int8) % 16) return fail(PTQ_ERR_ALIGN, "q must be 16-byte aligned");
+    if (reinterpret_cast<uintptr_t>(y_fp16) % 2) return fail(PTQ_ERR_ALIGN, "y must be 2-byte aligned");
+    ptq_status_t st = check_device(h);
+    if (st != PTQ_OK) return st;
+    const long long M = static_cast<long long>(B) * h->T;
+    if (ranges_overlap(q_int8, static_cast<size_t>(M) * h->Kpad, y_fp16, static_cast<size_t>(M) * h->N * 2))
+        return fail(PTQ_ERR_VALUE, "q and y overlap");
+    return launch_gemm(h, q_int8, M, y_fp16, nullptr, static_cast<cudaStream_t>(stream));
+}
+
 ptq_status_t ptq_linear_forward_debug(const ptq_linear_t *h, const void *x_fp16, int B, void *y_fp16,
                                       void *q_int8_out, void *acc_int32_out, void *workspace,
                                       size_t workspace_bytes, unsigned flags, void *stream)
