@@ -109,6 +109,33 @@ ptq_status_t ptq_linear_forward(const ptq_linear_t *h, const void *x_fp16, int B
                                 void *y_fp16, void *workspace, size_t workspace_bytes,
                                 unsigned flags, void *stream);
 
+/*
+ * Forward pass for callers that cannot allocate device memory.  (The paper has no counterpart of
+ * this entry point; it computes exactly what ptq_linear_forward with PTQ_FLAG_NONE computes.)
+ *
+ * Some callers have no way to provide the workspace: code running where cudaMalloc is forbidden
+ * (inside a latency-critical serving loop that must not touch the allocator, under a memory pool
+ * that owns every byte of the device, or in a plugin that is handed only its input and output
+ * buffers).  For them the int8 codes go to a scratch array that is part of the library image
+ * itself: a file-scope __device__ array of PTQ_STATIC_SCRATCH_BYTES bytes, present on every GPU
+ * that loads the library from load until process exit.
+ *
+ *   - B*T rows of ptq_linear_code_pitch(h) bytes must fit in PTQ_STATIC_SCRATCH_BYTES; larger
+ *     batches are refused with PTQ_ERR_SHAPE (split the batch, or use ptq_linear_forward).
+ *   - The call allocates nothing and frees nothing.  The first call on each device looks up the
+ *     array's device address (a one-time, per-device set-up step done with that device current);
+ *     make that first call before starting any stream capture.
+ *   - All calls on one device, from every handle and every stream, share the same array, and it
+ *     keeps whatever the previous call left in it.  Nothing in it needs to start at zero: each call
+ *     writes every byte it later reads.  Two calls whose GPU work overlaps in time (different
+ *     streams, no dependency between them) race on the array and corrupt each other's result; run
+ *     them on one stream or order them with events.
+ *   x_fp16, y_fp16, stream: as for ptq_linear_forward.
+ */
+#define PTQ_STATIC_SCRATCH_BYTES (32u * 1024u * 1024u)
+ptq_status_t ptq_linear_forward_static(const ptq_linear_t *h, const void *x_fp16, int B, void *y_fp16,
+                                       void *stream);
+
 /* 1 if PTQ_FLAG_FUSED_PROLOGUE runs the single fused kernel for this layer, 0 if it falls back. */
 int ptq_linear_fused_supported(const ptq_linear_t *h);
 

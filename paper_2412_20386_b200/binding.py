@@ -19,6 +19,7 @@ _SO = os.path.join(_HERE, "libptq_linear.so")
 
 FLAG_NONE = 0
 FLAG_FUSED_PROLOGUE = 1
+STATIC_SCRATCH_BYTES = 32 * 1024 * 1024
 
 _STATUS_NAMES = {0: "PTQ_OK", 1: "PTQ_ERR_NULL", 2: "PTQ_ERR_SHAPE", 3: "PTQ_ERR_VALUE",
                  4: "PTQ_ERR_ALIGN", 5: "PTQ_ERR_ARCH", 6: "PTQ_ERR_CUDA", 7: "PTQ_ERR_NOMEM",
@@ -56,6 +57,8 @@ def load_library() -> ctypes.CDLL:
     L.ptq_linear_workspace_bytes.argtypes = [vp, ci, cu]
     L.ptq_linear_forward.restype = ci
     L.ptq_linear_forward.argtypes = [vp, vp, ci, vp, vp, sz, cu, vp]
+    L.ptq_linear_forward_static.restype = ci
+    L.ptq_linear_forward_static.argtypes = [vp, vp, ci, vp, vp]
     L.ptq_linear_fused_supported.restype = ci
     L.ptq_linear_fused_supported.argtypes = [vp]
     L.ptq_quantize.restype = ci
@@ -172,6 +175,18 @@ class PtqLinear:
         wbytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
         _check(self._L.ptq_linear_forward(self._h, x.data_ptr(), B, y.data_ptr(), wptr, wbytes,
                                           flags, _stream_ptr(stream)))
+        return y
+
+    def forward_static(self, x, y, stream=None):
+        """``ptq_linear_forward_static``: forward pass that allocates nothing.
+
+        The caller passes both x and y; the int8 codes go to the scratch array built into the
+        library (at most ``STATIC_SCRATCH_BYTES``), which all calls on a device share.
+        """
+        B = self._batch(x)
+        if tuple(y.shape) != (B, self.T, self.N) or y.dtype != x.dtype or not y.is_contiguous() or not y.is_cuda:
+            raise ValueError("y must be a contiguous CUDA float16 tensor [B,T,N]")
+        _check(self._L.ptq_linear_forward_static(self._h, x.data_ptr(), B, y.data_ptr(), _stream_ptr(stream)))
         return y
 
     def quantize(self, x, q=None, stream=None):

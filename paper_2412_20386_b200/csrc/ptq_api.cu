@@ -243,6 +243,28 @@ ptq_status_t launch_gemm(const ptq_linear *h, const void *codes, long long M, vo
     return PTQ_OK;
 }
 
+// Scratch for ptq_linear_forward_static: lives in the library image on every device that loads it.
+// In host code the symbol below is only a stand-in; the kernels must be given the device address
+// that cudaGetSymbolAddress returns, looked up once per device with that device current.
+static __device__ __align__(256) unsigned char g_static_scratch[PTQ_STATIC_SCRATCH_BYTES];
+
+ptq_status_t static_scratch_address(int device, void **out)
+{
+    constexpr int kMaxDevices = 64;
+    static std::mutex mu;
+    static void *addr[kMaxDevices] = {};
+    if (device < 0 || device >= kMaxDevices) return fail(PTQ_ERR_CUDA, "device index %d out of range", device);
+    std::lock_guard<std::mutex> lock(mu);
+    if (!addr[device]) {
+        void *p = nullptr;
+        PTQ_CUDA(cudaGetSymbolAddress(&p, g_static_scratch));   // the current device is `device` (checked by the caller)
+        if (!p) return fail(PTQ_ERR_CUDA, "cudaGetSymbolAddress returned a null address");
+        addr[device] = p;
+    }
+    *out = addr[device];
+    return PTQ_OK;
+}
+
 ptq_status_t validate_forward(const ptq_linear *h, const void *x, int B, const void *y)
 {
     if (!h || !x || !y) return fail(PTQ_ERR_NULL, "handle, x and y must not be NULL");
@@ -460,6 +482,25 @@ ptq_status_t ptq_linear_forward(const ptq_linear_t *h, const void *x_fp16, int B
                                 size_t workspace_bytes, unsigned flags, void *stream)
 {
     return ptq_linear_forward_debug(h, x_fp16, B, y_fp16, nullptr, nullptr, workspace, workspace_bytes, flags, stream);
+}
+
+ptq_status_t ptq_linear_forward_static(const ptq_linear_t *h, const void *x_fp16, int B, void *y_fp16,
+                                       void *stream)
+{
+    ptq_status_t st = validate_forward(h, x_fp16, B, y_fp16);
+    if (st != PTQ_OK) return st;
+    const long long M = static_cast<long long>(B) * h->T;
+    const unsigned long long need = static_cast<unsigned long long>(M) * h->Kpad;
+    if (need > PTQ_STATIC_SCRATCH_BYTES)
+        return fail(PTQ_ERR_SHAPE,
+                    "B*T*pitch = %llu bytes of codes exceed the built-in scratch of %u bytes; "
+                    "split the batch or use ptq_linear_forward with a caller workspace",
+                    need, PTQ_STATIC_SCRATCH_BYTES);
+    void *scratch = nullptr;
+    if ((st = static_scratch_address(h->device, &scratch)) != PTQ_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if ((st = launch_quantize(h, x_fp16, M, scratch, h->Kpad, s)) != PTQ_OK) return st;
+    return launch_gemm(h, scratch, M, y_fp16, nullptr, s);
 }
 
 ptq_status_t ptq_linear_device_status(const ptq_linear_t *h)
