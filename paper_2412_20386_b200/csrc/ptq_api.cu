@@ -16,6 +16,7 @@
 #include <vector>
 
 #include "ptq_calibrate.cuh"
+#include "ptq_fused.cuh"
 #include "ptq_gemm.cuh"
 #include "ptq_quantize.cuh"
 
@@ -109,8 +110,13 @@ struct ptq_linear {
     float *d_dw = nullptr, *d_bias = nullptr;            // [n_tiles*BN rounded up to 64, +64], zero padded
     float *d_s = nullptr, *d_rs = nullptr;               // [round_up(K,16)]
     float *d_dx = nullptr, *d_rdx = nullptr;             // [T]
+    float2 *d_dx2 = nullptr;                             // [T] {dx, 1/dx}
     unsigned *d_status = nullptr;
     CUtensorMap tmW;
+    // A-stationary kernel (fused, and the two-kernel path's GEMM when the code panel fits shared memory)
+    bool as_ok = false;
+    int as_BN = 0, as_n_tiles = 0, as_w_stages = 0, as_w_stage_bytes = 0, as_staging = 0, as_smem = 0;
+    CUtensorMap tmWas;
 };
 
 namespace {
@@ -150,27 +156,37 @@ ptq_status_t launch_quantize(const ptq_linear *h, const void *x, long long M, vo
     p.rs = h->d_rs;
     p.dx = h->d_dx;
     p.rdx = h->d_rdx;
+    p.dx2 = h->d_dx2;
     p.M = M;
     p.K = h->K;
     p.T = h->T;
     p.q_pitch = q_pitch;
-    p.rows_per_iter = 0;
-    const bool vec = (h->K % 16 == 0) && (reinterpret_cast<uintptr_t>(x) % 16 == 0) &&
-                     (reinterpret_cast<uintptr_t>(q) % 16 == 0) && (q_pitch % 16 == 0);
+    const long long B = M / h->T;
+    // Vector kernel: thread count = S * (chunks per image), S images apart between a thread's chunks.
+    // S is the multiple of `mult` (which makes the thread count a multiple of 256) that brings the grid
+    // closest to one resident wave without exceeding it; shapes for which even the smallest S
+    // overshoots the wave by far go to the scalar kernel.
+    bool vec = (h->K % 8 == 0) && (reinterpret_cast<uintptr_t>(x) % 16 == 0) &&
+               (reinterpret_cast<uintptr_t>(q) % 8 == 0) && (q_pitch % 8 == 0);
+    long long cpi = 0, S = 0;
     if (vec) {
-        const int cpr = h->K / 16;
-        const int mult = cpr / gcd_int(cpr, 256);             // grid must make threads a multiple of cpr
-        const long long chunks = M * cpr;
-        long long want = (chunks + 511) / 512;                // two rows per thread per trip
-        const long long cap = static_cast<long long>(h->num_sms) * 6;
-        if (want > cap) want = cap;
-        if (want < 1) want = 1;
-        const int grid = round_up(static_cast<int>(want), mult);
-        p.rows_per_iter = grid * 256 / cpr;
+        cpi = static_cast<long long>(h->T) * (h->K / 8);
+        const long long wave = static_cast<long long>(h->num_sms) * ptq::kQuantCtasPerSm * 256;
+        const long long mult = 256 / gcd_int(static_cast<int>(cpi % 256 == 0 ? 256 : cpi % 256), 256);
+        S = wave / cpi / mult * mult;
+        if (S < mult) S = mult;
+        const long long bcap = (B + mult - 1) / mult * mult;      // more than B images apart is idle threads only
+        if (S > bcap) S = bcap;
+        if (S * cpi > 4 * wave) vec = false;
+    }
+    p.B = static_cast<int>(B);
+    p.imgs_per_iter = static_cast<int>(S);
+    if (vec) {
+        const int grid = static_cast<int>(S * cpi / 256);
         if (h->fast_div)
-            ptq::ptq_quantize_vec16_kernel<true><<<grid, 256, 0, stream>>>(p);
+            ptq::ptq_quantize_vec8_kernel<true><<<grid, 256, 0, stream>>>(p);
         else
-            ptq::ptq_quantize_vec16_kernel<false><<<grid, 256, 0, stream>>>(p);
+            ptq::ptq_quantize_vec8_kernel<false><<<grid, 256, 0, stream>>>(p);
     } else {
         long long want = (M * h->K + 255) / 256;
         const long long cap = static_cast<long long>(h->num_sms) * 8;
@@ -231,6 +247,7 @@ ptq_status_t launch_gemm(const ptq_linear *h, const void *codes, long long M, vo
     p.status = h->d_status;
     p.use_tma_store = tma_store ? 1 : 0;
     p.y_vec2 = (h->N % 2 == 0 && reinterpret_cast<uintptr_t>(y) % 4 == 0) ? 1 : 0;
+    p.y_vec8 = 0;   // this kernel always has a staging buffer; 16-byte alignment means TMA stores
 
     const long long tiles = static_cast<long long>(p.m_tiles) * p.n_tiles;
     const int grid = static_cast<int>(tiles < h->num_sms ? tiles : h->num_sms);
@@ -242,6 +259,122 @@ ptq_status_t launch_gemm(const ptq_linear *h, const void *codes, long long M, vo
     PTQ_CUDA(cudaGetLastError());
     return PTQ_OK;
 }
+
+// Tiling of the A-stationary kernel for a layer: the code panel (k_blocks x 16 KB) stays resident, the
+// rest of shared memory holds weight stages and, if it fits, the epilogue's staging buffers.
+void choose_astat(ptq_linear *h)
+{
+    h->as_ok = false;
+    if (h->k_blocks > ptq::kFusedMaxKBlocks) return;
+    const int cand_bn[3] = {h->BN, 128, 64};
+    for (int staging = 1; staging >= 0 && !h->as_ok; --staging) {
+        for (int c = 0; c < 3 && !h->as_ok; ++c) {
+            int bn = cand_bn[c];
+            if (c > 0 && bn >= h->BN) continue;
+            const int n_tiles = (c == 0) ? h->n_tiles : (h->N + bn - 1) / bn;
+            const int stage_bytes = bn * ptq::kBK;
+            const int fixed = ptq::fused_smem_bytes(h->k_blocks, 0, 0, staging);
+            int stages = (ptq::kFusedSmemLimit - fixed) / stage_bytes;
+            if (stages < 2) continue;
+            if (stages > ptq::kFusedMaxWStages) stages = ptq::kFusedMaxWStages;
+            h->as_ok = true;
+            h->as_BN = bn;
+            h->as_n_tiles = n_tiles;
+            h->as_w_stages = stages;
+            h->as_w_stage_bytes = stage_bytes;
+            h->as_staging = staging;
+            h->as_smem = ptq::fused_smem_bytes(h->k_blocks, stages, stage_bytes, staging);
+        }
+    }
+}
+
+template <typename Kern>
+ptq_status_t launch_astat_kernel(Kern kern, int threads, const ptq_linear *h, const CUtensorMap &tmA,
+                                 const CUtensorMap &tmY, const ptq::FusedParams &fp, int grid, cudaStream_t stream)
+{
+    PTQ_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ptq::kFusedSmemLimit));
+    kern<<<grid, threads, h->as_smem, stream>>>(tmA, h->tmWas, tmY, fp);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    PTQ_CUDA(cudaGetLastError());
+    return PTQ_OK;
+}
+
+// A-stationary launch.  quantize = true: `src` is x fp16 [M,K] (Q1 + G1 + E1 in one kernel);
+// quantize = false: `src` is the code matrix [M,Kpad] (G1 + E1).
+ptq_status_t launch_astat(const ptq_linear *h, const void *src, bool quantize, long long M, void *y, void *acc_out,
+                          cudaStream_t stream)
+{
+    CUtensorMap tmA, tmY;
+    ptq_status_t st;
+    if (!quantize) {
+        st = make_map_2d(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, src, static_cast<unsigned long long>(h->K),
+                         static_cast<unsigned long long>(M), static_cast<unsigned long long>(h->Kpad), ptq::kBK,
+                         ptq::kBM);
+        if (st != PTQ_OK) return st;
+    } else {
+        tmA = h->tmWas;   // unused by the kernel in this mode
+    }
+    const bool aligned = (h->N % 8 == 0) && (reinterpret_cast<uintptr_t>(y) % 16 == 0);
+    const bool tma_store = aligned && h->as_staging;
+    if (tma_store) {
+        st = make_map_2d(&tmY, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, y, static_cast<unsigned long long>(h->N),
+                         static_cast<unsigned long long>(M), static_cast<unsigned long long>(h->N) * 2,
+                         ptq::kStoreBoxCols, 32);
+        if (st != PTQ_OK) return st;
+    } else {
+        tmY = h->tmWas;
+    }
+    ptq::FusedParams fp;
+    ptq::GemmParams &p = fp.g;
+    p.M = M;
+    p.N = h->N;
+    p.K = h->K;
+    p.T = h->T;
+    p.BN = h->as_BN;
+    p.n_tiles = h->as_n_tiles;
+    p.m_tiles = static_cast<int>((M + ptq::kBM - 1) / ptq::kBM);
+    p.k_blocks = h->k_blocks;
+    p.last_mmas = h->last_mmas;
+    p.dx = h->d_dx;
+    p.dw = h->d_dw;
+    p.bias = h->d_bias;
+    p.y = static_cast<__half *>(y);
+    p.acc_out = static_cast<int32_t *>(acc_out);
+    p.status = h->d_status;
+    p.use_tma_store = tma_store ? 1 : 0;
+    p.y_vec2 = (h->N % 2 == 0 && reinterpret_cast<uintptr_t>(y) % 4 == 0) ? 1 : 0;
+    p.y_vec8 = (aligned && !tma_store) ? 1 : 0;
+    fp.x = static_cast<const __half *>(quantize ? src : nullptr);
+    fp.s = h->d_s;
+    fp.rs = h->d_rs;
+    fp.dx2 = h->d_dx2;
+    fp.w_stages = h->as_w_stages;
+    fp.w_stage_bytes = h->as_w_stage_bytes;
+    fp.has_staging = h->as_staging;
+    const int grid = p.m_tiles < h->num_sms ? p.m_tiles : h->num_sms;
+    const bool dbg = acc_out != nullptr;
+    if (quantize) {
+        const int th = ptq::kFusedThreadsQuant;
+        if (h->fast_div)
+            return dbg ? launch_astat_kernel(ptq::ptq_fused_linear_kernel<true, true, true>, th, h, tmA, tmY, fp, grid, stream)
+                       : launch_astat_kernel(ptq::ptq_fused_linear_kernel<true, true, false>, th, h, tmA, tmY, fp, grid, stream);
+        return dbg ? launch_astat_kernel(ptq::ptq_fused_linear_kernel<true, false, true>, th, h, tmA, tmY, fp, grid, stream)
+                   : launch_astat_kernel(ptq::ptq_fused_linear_kernel<true, false, false>, th, h, tmA, tmY, fp, grid, stream);
+    }
+    const int th = ptq::kFusedThreadsPlain;
+    return dbg ? launch_astat_kernel(ptq::ptq_fused_linear_kernel<false, true, true>, th, h, tmA, tmY, fp, grid, stream)
+               : launch_astat_kernel(ptq::ptq_fused_linear_kernel<false, true, false>, th, h, tmA, tmY, fp, grid, stream);
+}
+
+// G1 + E1 on codes: the A-stationary kernel when the layer's code panel fits, else the streaming one.
+ptq_status_t launch_gemm_any(const ptq_linear *h, const void *codes, long long M, void *y, void *acc_out,
+                             cudaStream_t stream)
+{
+    if (h->as_ok) return launch_astat(h, codes, false, M, y, acc_out, stream);
+    return launch_gemm(h, codes, M, y, acc_out, stream);
+}
+
+bool fused_usable(const ptq_linear *h) { return h->as_ok && h->K % 16 == 0; }
 
 // Scratch for ptq_linear_forward_static: lives in the library image on every device that loads it.
 // In host code the symbol below is only a stand-in; the kernels must be given the device address
@@ -312,6 +445,7 @@ void ptq_linear_destroy(ptq_linear_t *h)
     cudaFree(h->d_rs);
     cudaFree(h->d_dx);
     cudaFree(h->d_rdx);
+    cudaFree(h->d_dx2);
     cudaFree(h->d_status);
     delete h;
 }
@@ -374,7 +508,9 @@ ptq_status_t ptq_linear_create(ptq_linear_t **out, int K, int N, int T, const in
     h->k_blocks = (K + ptq::kBK - 1) / ptq::kBK;
     h->last_mmas = (K - (h->k_blocks - 1) * ptq::kBK + 31) / 32;
 
-    const int Npad = h->n_tiles * h->BN;
+    choose_astat(h);
+    int Npad = h->n_tiles * h->BN;
+    if (h->as_ok && h->as_n_tiles * h->as_BN > Npad) Npad = h->as_n_tiles * h->as_BN;
     const int Nvec = round_up(Npad, 64) + 64;
     const int Kvec = round_up(K, 16);
     std::vector<int8_t> wpad(static_cast<size_t>(Npad) * h->Kpad, 0);
@@ -384,7 +520,12 @@ ptq_status_t ptq_linear_create(ptq_linear_t **out, int K, int N, int T, const in
         sp[k] = smooth[k];
         rs[k] = 1.0f / smooth[k];
     }
-    for (int t = 0; t < T; ++t) rdx[t] = 1.0f / act_step[t];
+    std::vector<float> dx2(2 * static_cast<size_t>(T));
+    for (int t = 0; t < T; ++t) {
+        rdx[t] = 1.0f / act_step[t];
+        dx2[2 * t] = act_step[t];
+        dx2[2 * t + 1] = rdx[t];
+    }
 
     ptq_status_t st = PTQ_OK;
     do {
@@ -395,10 +536,18 @@ ptq_status_t ptq_linear_create(ptq_linear_t **out, int K, int N, int T, const in
         if ((st = upload(reinterpret_cast<void **>(&h->d_rs), rs.data(), sizeof(float) * Kvec, sizeof(float) * Kvec)) != PTQ_OK) break;
         if ((st = upload(reinterpret_cast<void **>(&h->d_dx), act_step, sizeof(float) * T, sizeof(float) * T)) != PTQ_OK) break;
         if ((st = upload(reinterpret_cast<void **>(&h->d_rdx), rdx.data(), sizeof(float) * T, sizeof(float) * T)) != PTQ_OK) break;
+        if ((st = upload(reinterpret_cast<void **>(&h->d_dx2), dx2.data(), sizeof(float) * 2 * T, sizeof(float) * 2 * T)) != PTQ_OK) break;
         if ((st = upload(reinterpret_cast<void **>(&h->d_status), nullptr, 0, sizeof(unsigned))) != PTQ_OK) break;
         st = make_map_2d(&h->tmW, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, h->d_w, static_cast<unsigned long long>(K),
                          static_cast<unsigned long long>(Npad), static_cast<unsigned long long>(h->Kpad), ptq::kBK,
                          static_cast<unsigned>(h->BN));
+        if (st != PTQ_OK) break;
+        if (h->as_ok)
+            st = make_map_2d(&h->tmWas, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, h->d_w, static_cast<unsigned long long>(K),
+                             static_cast<unsigned long long>(Npad), static_cast<unsigned long long>(h->Kpad),
+                             ptq::kBK, static_cast<unsigned>(h->as_BN));
+        else
+            h->tmWas = h->tmW;
     } while (0);
     if (st != PTQ_OK) {
         char keep[sizeof(g_err)];
@@ -418,11 +567,7 @@ size_t ptq_linear_workspace_bytes(const ptq_linear_t *h, int B, unsigned flags)
     return static_cast<size_t>(B) * h->T * h->Kpad;
 }
 
-int ptq_linear_fused_supported(const ptq_linear_t *h)
-{
-    (void)h;
-    return 0;
-}
+int ptq_linear_fused_supported(const ptq_linear_t *h) { return (h && fused_usable(h)) ? 1 : 0; }
 
 ptq_status_t ptq_quantize(const ptq_linear_t *h, const void *x_fp16, int B, void *q_int8, void *stream)
 {
@@ -450,7 +595,7 @@ ptq_status_t ptq_linear_gemm_dequant(const ptq_linear_t *h, const void *q_int8, 
     const long long M = static_cast<long long>(B) * h->T;
     if (ranges_overlap(q_int8, static_cast<size_t>(M) * h->Kpad, y_fp16, static_cast<size_t>(M) * h->N * 2))
         return fail(PTQ_ERR_VALUE, "q and y overlap");
-    return launch_gemm(h, q_int8, M, y_fp16, nullptr, static_cast<cudaStream_t>(stream));
+    return launch_gemm_any(h, q_int8, M, y_fp16, nullptr, static_cast<cudaStream_t>(stream));
 }
 
 ptq_status_t ptq_linear_forward_debug(const ptq_linear_t *h, const void *x_fp16, int B, void *y_fp16,
@@ -462,8 +607,15 @@ ptq_status_t ptq_linear_forward_debug(const ptq_linear_t *h, const void *x_fp16,
     if (flags & ~PTQ_FLAG_FUSED_PROLOGUE) return fail(PTQ_ERR_VALUE, "unknown flags 0x%x", flags);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const long long M = static_cast<long long>(B) * h->T;
+    if ((flags & PTQ_FLAG_FUSED_PROLOGUE) && fused_usable(h) && reinterpret_cast<uintptr_t>(x_fp16) % 16 == 0) {
+        // F1: one kernel, no workspace.  The codes never exist in memory; a requested tap is produced by
+        // the quantize kernel on its own.
+        if ((st = launch_astat(h, x_fp16, true, M, y_fp16, acc_int32_out, s)) != PTQ_OK) return st;
+        if (q_int8_out) return launch_quantize(h, x_fp16, M, q_int8_out, h->K, s);
+        return PTQ_OK;
+    }
     const size_t need = static_cast<size_t>(M) * h->Kpad;
-    if (!workspace) return fail(PTQ_ERR_NULL, "workspace must not be NULL for this layer and these flags");
+    if (!workspace) return fail(PTQ_ERR_NULL, "workspace must not be NULL for this layer, alignment and flags");
     if (workspace_bytes < need)
         return fail(PTQ_ERR_SHAPE, "workspace has %zu bytes, %zu needed", workspace_bytes, need);
     if (reinterpret_cast<uintptr_t>(workspace) % 16) return fail(PTQ_ERR_ALIGN, "workspace must be 16-byte aligned");
@@ -471,7 +623,7 @@ ptq_status_t ptq_linear_forward_debug(const ptq_linear_t *h, const void *x_fp16,
         ranges_overlap(workspace, need, x_fp16, static_cast<size_t>(M) * h->K * 2))
         return fail(PTQ_ERR_VALUE, "workspace overlaps x or y");
     if ((st = launch_quantize(h, x_fp16, M, workspace, h->Kpad, s)) != PTQ_OK) return st;
-    if ((st = launch_gemm(h, workspace, M, y_fp16, acc_int32_out, s)) != PTQ_OK) return st;
+    if ((st = launch_gemm_any(h, workspace, M, y_fp16, acc_int32_out, s)) != PTQ_OK) return st;
     if (q_int8_out)
         PTQ_CUDA(cudaMemcpy2DAsync(q_int8_out, h->K, workspace, h->Kpad, h->K, static_cast<size_t>(M),
                                    cudaMemcpyDeviceToDevice, s));
@@ -500,7 +652,7 @@ ptq_status_t ptq_linear_forward_static(const ptq_linear_t *h, const void *x_fp16
     if ((st = static_scratch_address(h->device, &scratch)) != PTQ_OK) return st;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if ((st = launch_quantize(h, x_fp16, M, scratch, h->Kpad, s)) != PTQ_OK) return st;
-    return launch_gemm(h, scratch, M, y_fp16, nullptr, s);
+    return launch_gemm_any(h, scratch, M, y_fp16, nullptr, s);
 }
 
 ptq_status_t ptq_linear_device_status(const ptq_linear_t *h)

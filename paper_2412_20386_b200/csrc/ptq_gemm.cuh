@@ -7,13 +7,14 @@
 // The rank-1 scaling is applied to the accumulator as it leaves TMEM, so neither the int32
 // product nor an [M,N] step-size tensor ever reaches HBM.
 //
-// One persistent CTA per SM, 6 warps:
+// One persistent CTA per SM, 10 warps:
 //   warp 0      TMA producer: A tile 128 x 128 B of codes and B tile BN x 128 B of weights per
 //               stage, both written with the 128-byte swizzle, completion on a "full" mbarrier
 //   warp 1      owns TMEM (512 columns = two 128 x 256 accumulators) and issues the MMAs; a
 //               tcgen05.commit frees each shared-memory stage and publishes each accumulator
-//   warps 2..5  epilogue: tcgen05.ld (each warp its own 32-lane quarter), scale, convert, stage the
-//               fp16 tile in swizzled shared memory and write it with a TMA store
+//   warps 2..9  epilogue: tcgen05.ld (lane quarter = warp % 4; the two warps of a quarter take
+//               alternate 64-column boxes), scale, convert, stage the fp16 box in swizzled shared
+//               memory and write it with a TMA store
 // While the epilogue drains accumulator i the MMA warp already fills accumulator i^1.
 #pragma once
 
@@ -31,10 +32,10 @@ constexpr int kStages = 4;
 constexpr int kATileBytes = kBM * kBK;                    // 16 KB
 constexpr int kBTileBytes = kMaxBN * kBK;                 // 32 KB
 constexpr int kStageBytes = kATileBytes + kBTileBytes;
-constexpr int kNumEpiWarps = 4;
+constexpr int kNumEpiWarps = 8;                           // two per TMEM lane quarter
 constexpr int kStoreBoxCols = 64;                         // fp16 columns per TMA store box (128 B)
 constexpr int kStoreBoxBytes = 32 * kStoreBoxCols * 2;    // 32 rows x 128 B
-constexpr int kStagingBytesPerWarp = 2 * kStoreBoxBytes;  // double buffered
+constexpr int kStagingBytesPerWarp = kStoreBoxBytes;      // reused once the previous box has been read
 constexpr int kGemmThreads = 32 * (2 + kNumEpiWarps);
 constexpr int kTmemCols = 512;
 constexpr int kNumBarriers = 2 * kStages + 4;
@@ -56,6 +57,7 @@ struct GemmParams {
     unsigned *status;  // device status word
     int use_tma_store; // y is written by TMA (needs N % 8 == 0 and a 16-byte aligned y)
     int y_vec2;        // plain-store path may use 4-byte stores (N even, y 4-byte aligned)
+    int y_vec8;        // plain-store path may use 16-byte stores (N % 8 == 0, y 16-byte aligned)
 };
 
 // --- epilogue helpers -------------------------------------------------------------------------
@@ -120,6 +122,28 @@ __device__ __forceinline__ void convert_store32_plain(const uint32_t (&v)[32], f
     }
 }
 
+// 16-byte stores of 32 columns of this thread's row straight from registers (N % 8 == 0 and a
+// 16-byte aligned y): the thread's 64 contiguous bytes go out as four stores that L2 merges.
+__device__ __forceinline__ void convert_store32_vec8(const uint32_t (&v)[32], float dxr, const float *dw,
+                                                     const float *bias, __half *yrow, int n_first, int N)
+{
+#pragma unroll
+    for (int jj = 0; jj < 4; ++jj) {
+        const int n = n_first + 8 * jj;
+        if (n >= N) break;
+        const float4 w0 = __ldg(reinterpret_cast<const float4 *>(dw + 8 * jj));
+        const float4 w1 = __ldg(reinterpret_cast<const float4 *>(dw + 8 * jj + 4));
+        const float4 b0 = __ldg(reinterpret_cast<const float4 *>(bias + 8 * jj));
+        const float4 b1 = __ldg(reinterpret_cast<const float4 *>(bias + 8 * jj + 4));
+        uint4 o;
+        o.x = pack_half2(dequant_one(v[8 * jj + 0], dxr, w0.x, b0.x), dequant_one(v[8 * jj + 1], dxr, w0.y, b0.y));
+        o.y = pack_half2(dequant_one(v[8 * jj + 2], dxr, w0.z, b0.z), dequant_one(v[8 * jj + 3], dxr, w0.w, b0.w));
+        o.z = pack_half2(dequant_one(v[8 * jj + 4], dxr, w1.x, b1.x), dequant_one(v[8 * jj + 5], dxr, w1.y, b1.y));
+        o.w = pack_half2(dequant_one(v[8 * jj + 6], dxr, w1.z, b1.z), dequant_one(v[8 * jj + 7], dxr, w1.w, b1.w));
+        *reinterpret_cast<uint4 *>(yrow + n) = o;
+    }
+}
+
 __device__ __forceinline__ void store_acc32(const uint32_t (&v)[32], int32_t *arow, int n_first, int N)
 {
 #pragma unroll
@@ -132,11 +156,11 @@ __device__ __forceinline__ void store_acc32(const uint32_t (&v)[32], int32_t *ar
 template <bool kDebugAcc>
 __device__ __forceinline__ uint32_t epilogue_tile(const GemmParams &p, const CUtensorMap *tmY, uint32_t tmem_row,
                                                   long long m_row0, int n0, float dxr, uint32_t staging,
-                                                  uint32_t nboxes, int lane)
+                                                  uint32_t nboxes, int lane, int col_half)
 {
     const long long m = m_row0 + lane;
     const bool row_ok = m < p.M;
-    for (int c0 = 0; c0 < p.BN; c0 += kStoreBoxCols) {
+    for (int c0 = col_half * kStoreBoxCols; c0 < p.BN; c0 += 2 * kStoreBoxCols) {
         uint32_t v0[32], v1[32];
         tmem_ld_32x32(tmem_row + c0, v0);
         tmem_ld_32x32(tmem_row + c0 + 32, v1);
@@ -149,8 +173,8 @@ __device__ __forceinline__ uint32_t epilogue_tile(const GemmParams &p, const CUt
             }
         }
         if (p.use_tma_store) {
-            const uint32_t buf = staging + (nboxes & 1u) * kStoreBoxBytes;
-            if (nboxes >= 2u && lane == 0) bulk_wait_group_read<1>();   // the box that used this buffer was read
+            const uint32_t buf = staging;
+            if (nboxes >= 1u && lane == 0) bulk_wait_group_read<0>();   // the previous box has left the buffer
             __syncwarp();
             const uint32_t row_addr = buf + static_cast<uint32_t>(lane) * 128u;
             convert_stage32(v0, 0, dxr, p.dw + n_first, p.bias + n_first, row_addr, lane);
@@ -163,6 +187,10 @@ __device__ __forceinline__ uint32_t epilogue_tile(const GemmParams &p, const CUt
                 bulk_commit_group();
             }
             ++nboxes;
+        } else if (row_ok && p.y_vec8) {
+            __half *yrow = p.y + m * p.N;
+            convert_store32_vec8(v0, dxr, p.dw + n_first, p.bias + n_first, yrow, n_first, p.N);
+            convert_store32_vec8(v1, dxr, p.dw + n_first + 32, p.bias + n_first + 32, yrow, n_first + 32, p.N);
         } else if (row_ok) {
             __half *yrow = p.y + m * p.N;
             convert_store32_plain(v0, dxr, p.dw + n_first, p.bias + n_first, yrow, n_first, p.N, p.y_vec2 != 0);
@@ -295,6 +323,7 @@ ptq_gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     } else {
         // ------------------------------------------------------------------ epilogue warps
         const int quarter = warp & 3;                // TMEM lanes [32*quarter, 32*quarter+32)
+        const int col_half = (warp - 2) >> 2;        // which of the alternating 64-column boxes
         const uint32_t staging = staging_base + static_cast<uint32_t>(warp - 2) * kStagingBytesPerWarp;
         uint32_t buf = 0, bphase = 0, nboxes = 0;
         for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
@@ -308,7 +337,7 @@ ptq_gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             if (!got) break;
             tc_fence_after_sync();
             const uint32_t tmem_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * kMaxBN;
-            nboxes = epilogue_tile<kDebugAcc>(p, &tmY, tmem_row, m_row0, n_tile * p.BN, dxr, staging, nboxes, lane);
+            nboxes = epilogue_tile<kDebugAcc>(p, &tmY, tmem_row, m_row0, n_tile * p.BN, dxr, staging, nboxes, lane, col_half);
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(tempty_bar(buf));

@@ -48,47 +48,75 @@ __device__ __forceinline__ int quantize_fast(float xf, float s, float rs, float 
     return f32_to_code(div_rn_by_reciprocal(u, dx, rdx));
 }
 
-// True if either binary16 half of w has all exponent bits set (inf or NaN).
-__device__ __forceinline__ bool half2_has_nonfinite(uint32_t w)
-{
-    const uint32_t t = (w & 0x7c007c00u) + 0x04000400u;   // 0x7c00 + 0x0400 carries into bit 15
-    return (t & 0x80008000u) != 0u;
-}
-
 __device__ __forceinline__ uint32_t pack4(int a, int b, int c, int d)
 {
-    return (static_cast<uint32_t>(a) & 0xffu) | ((static_cast<uint32_t>(b) & 0xffu) << 8) |
-           ((static_cast<uint32_t>(c) & 0xffu) << 16) | (static_cast<uint32_t>(d) << 24);
+    // low bytes of four registers -> one word (a lowest)
+    const uint32_t ab = __byte_perm(static_cast<uint32_t>(a), static_cast<uint32_t>(b), 0x0040);
+    const uint32_t cd = __byte_perm(static_cast<uint32_t>(c), static_cast<uint32_t>(d), 0x0040);
+    return __byte_perm(ab, cd, 0x5410);
 }
 
-// Quantize 8 consecutive channels held as 4 packed half2 words into 2 words of codes.
-// s8 / rs8 point at the 8 channels' s and RN(1/s).
-template <bool kFast>
-__device__ __forceinline__ void quantize8(uint32_t x0, uint32_t x1, uint32_t x2, uint32_t x3, const float *s8,
-                                          const float *rs8, float dx, float rdx, uint32_t &lo, uint32_t &hi)
+// Screening threshold of the fast route below.  v' = x * (RN(1/s) * RN(1/dx)) differs from the
+// defined value v = RN(RN(x/s)/dx) by six roundings: |v' - v| <= 6 * 2^-24 * (1 + tiny) * |v|, which is
+// below 4.6e-5 for |v| <= 127.5, the largest magnitude at which a rounding tie still changes the
+// clamped code.  If v' is farther than 6e-5 from every half-integer, rint(v') = rint(v).
+constexpr float kScreenThreshold = 0.49994f;
+constexpr float kRoundMagic = 12582912.0f;   // 1.5 * 2^23: (v + magic) - magic = rint(v) for |v| < 2^22
+
+// |v - rint(v)| for |v| < 2^22; NaN for NaN and infinite v; meaningless (but finite or NaN) beyond.
+__device__ __forceinline__ float dist_to_integer(float v)
+{
+    const float r = __fadd_rn(__fadd_rn(v, kRoundMagic), -kRoundMagic);
+    return fabsf(__fadd_rn(v, -r));
+}
+
+// Fast route for 8 consecutive channels held as 4 packed half2 words: one multiply by the combined
+// reciprocal c = RN(RN(1/s) * RN(1/dx)), the saturating round-to-nearest-even conversion, and a
+// distance-to-tie test.  Returns true when one of the 8 values sits within the error bound of a
+// rounding tie, in which case the caller recomputes the 8 codes with the two exact divisions.
+// Values beyond +-127.5 clamp to the same code whichever way a tie falls, NaN converts to 0 and
+// infinities saturate on both routes, so a needless trip through the exact route (NaN, inf and huge
+// values fail the test) costs time only: the final codes are always those of the definition.
+// Valid only when every scale lies in [2^-30, 2^30] (no under/overflow in c or x * c).
+__device__ __forceinline__ bool quantize8_screen(uint32_t x0, uint32_t x1, uint32_t x2, uint32_t x3,
+                                                 const float (&c8)[8], uint32_t &lo, uint32_t &hi)
 {
     const uint32_t xw[4] = {x0, x1, x2, x3};
     int c[8];
-    bool slow = !kFast;
-    if (kFast)
-        slow = half2_has_nonfinite(x0) || half2_has_nonfinite(x1) || half2_has_nonfinite(x2) ||
-               half2_has_nonfinite(x3);
-    if (slow) {
+    bool near_tie = false;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            __half2 h = *reinterpret_cast<const __half2 *>(&xw[i]);
-            const float2 f = __half22float2(h);
-            c[2 * i] = quantize_ieee(f.x, s8[2 * i], dx);
-            c[2 * i + 1] = quantize_ieee(f.y, s8[2 * i + 1], dx);
-        }
-    } else {
+    for (int i = 0; i < 4; ++i) {
+        __half2 h = *reinterpret_cast<const __half2 *>(&xw[i]);
+        const float2 f = __half22float2(h);
+        const float v0 = __fmul_rn(f.x, c8[2 * i]);
+        const float v1 = __fmul_rn(f.y, c8[2 * i + 1]);
+        c[2 * i] = f32_to_code(v0);
+        c[2 * i + 1] = f32_to_code(v1);
+        near_tie = near_tie || !(dist_to_integer(v0) <= kScreenThreshold);
+        near_tie = near_tie || !(dist_to_integer(v1) <= kScreenThreshold);
+    }
+    lo = pack4(c[0], c[1], c[2], c[3]);
+    hi = pack4(c[4], c[5], c[6], c[7]);
+    return near_tie;
+}
+
+// Exact route for the same 8 channels: two correctly rounded divisions per element.  s8 / rs8 point
+// at the channels' s and RN(1/s) in global memory.
+template <bool kFast>
+__device__ __noinline__ void quantize8_exact(uint32_t x0, uint32_t x1, uint32_t x2, uint32_t x3, const float *s8,
+                                             const float *rs8, float dx, float rdx, uint32_t &lo, uint32_t &hi)
+{
+    const uint32_t xw[4] = {x0, x1, x2, x3};
+    int c[8];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            __half2 h = *reinterpret_cast<const __half2 *>(&xw[i]);
-            const float2 f = __half22float2(h);
-            c[2 * i] = quantize_fast(f.x, s8[2 * i], rs8[2 * i], dx, rdx);
-            c[2 * i + 1] = quantize_fast(f.y, s8[2 * i + 1], rs8[2 * i + 1], dx, rdx);
-        }
+    for (int i = 0; i < 8; ++i) {
+        const __half hv = __ushort_as_half(static_cast<unsigned short>(xw[i >> 1] >> ((i & 1) * 16)));
+        const float f = __half2float(hv);
+        const float sv = __ldg(s8 + i);
+        if (kFast && fabsf(f) <= 65504.0f)
+            c[i] = quantize_fast(f, sv, __ldg(rs8 + i), dx, rdx);
+        else
+            c[i] = quantize_ieee(f, sv, dx);
     }
     lo = pack4(c[0], c[1], c[2], c[3]);
     hi = pack4(c[4], c[5], c[6], c[7]);
@@ -101,72 +129,89 @@ struct QuantParams {
     const float *rs;     // [K]  RN(1/s)
     const float *dx;     // [T]
     const float *rdx;    // [T]  RN(1/dx)
+    const float2 *dx2;   // [T]  {dx, RN(1/dx)} interleaved (one 8-byte load)
     long long M;
     int K;
     int T;
     int q_pitch;         // bytes between rows of q
-    int rows_per_iter;   // vector kernel: rows advanced per grid-stride step (grid threads / chunks per row)
+    int B;               // images (M = B * T)
+    int imgs_per_iter;   // vector kernel: images between consecutive chunks of one thread
 };
 
-// Vector path: K % 16 == 0, x and q 16-byte aligned, q_pitch % 16 == 0.
-// A "chunk" is 16 consecutive channels of one row: 2 x 16-byte loads, 1 x 16-byte store.
-// The grid's thread count is a multiple of the chunks per row, so each thread keeps the same 16
-// channels for the whole launch and holds their s and 1/s in registers.
-template <bool kFast>
-__global__ void __launch_bounds__(256) ptq_quantize_vec16_kernel(QuantParams p)
-{
-    const int cpr = p.K >> 4;                                        // chunks per row
-    const long long gtid = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
-    const int kc = static_cast<int>(gtid % cpr);
-    long long row = gtid / cpr;
-    int t = static_cast<int>(row % p.T);
-    const int t_step = p.rows_per_iter % p.T;
+#ifndef PTQ_QUANT_CTAS_PER_SM
+#define PTQ_QUANT_CTAS_PER_SM 4
+#endif
+#ifndef PTQ_QUANT_IMGS_PER_TRIP
+#define PTQ_QUANT_IMGS_PER_TRIP 2
+#endif
+constexpr int kQuantCtasPerSm = PTQ_QUANT_CTAS_PER_SM;     // resident CTAs per SM the vector kernel is built and launched for
+constexpr int kQuantImgsPerTrip = PTQ_QUANT_IMGS_PER_TRIP; // 16-byte loads per thread and trip (twice that in flight with the prefetch)
 
-    float s16[16], rs16[16];
-    {
-        const float4 *sp = reinterpret_cast<const float4 *>(p.s + kc * 16);
-        const float4 *rp = reinterpret_cast<const float4 *>(p.rs + kc * 16);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const float4 a = __ldg(sp + i), b = __ldg(rp + i);
-            s16[4 * i] = a.x; s16[4 * i + 1] = a.y; s16[4 * i + 2] = a.z; s16[4 * i + 3] = a.w;
-            rs16[4 * i] = b.x; rs16[4 * i + 1] = b.y; rs16[4 * i + 2] = b.z; rs16[4 * i + 3] = b.w;
-        }
+// Vector path: K % 8 == 0, x 16-byte aligned, q 8-byte aligned, q_pitch % 8 == 0.
+// A "chunk" is 8 consecutive channels of one token row: one 16-byte load, one 8-byte store.
+// Thread g of the grid owns chunk (g mod chunks-per-image) of images b0, b0+S, b0+2S, ... with
+// b0 = g / chunks-per-image; the grid's thread count is S * chunks-per-image.  A thread therefore
+// sees ONE token position and ONE group of 8 channels for the whole launch -- that is what "static"
+// per-token steps buy: the 8 combined reciprocals RN(1/s[k]) * RN(1/dx[t]) are formed once and kept
+// in registers, and the per-element work is convert, multiply, round, tie test.  Consecutive lanes
+// take consecutive chunks, so warp-wide accesses are contiguous 512-byte loads and 256-byte stores.
+// Each trip converts kQuantImgsPerTrip chunks and issues the next trip's loads first.
+template <bool kFast>
+__global__ void __launch_bounds__(256, kQuantCtasPerSm) ptq_quantize_vec8_kernel(QuantParams p)
+{
+    constexpr int U = kQuantImgsPerTrip;
+    const int cpr = p.K >> 3;                                        // chunks per row
+    const int cpi = p.T * cpr;                                       // chunks per image
+    const long long gtid = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+    const int c = static_cast<int>(gtid % cpi);
+    int b = static_cast<int>(gtid / cpi);
+    const int t = c / cpr;
+    const int kc = c - t * cpr;
+    const int S = p.imgs_per_iter;
+
+    const float2 d = __ldg(p.dx2 + t);
+    const float *s8 = p.s + kc * 8;          // read only on the exact route
+    const float *rs8 = p.rs + kc * 8;
+    float c8[8];
+    if (kFast) {
+        const float4 r0 = __ldg(reinterpret_cast<const float4 *>(rs8));
+        const float4 r1 = __ldg(reinterpret_cast<const float4 *>(rs8) + 1);
+        c8[0] = __fmul_rn(r0.x, d.y); c8[1] = __fmul_rn(r0.y, d.y); c8[2] = __fmul_rn(r0.z, d.y); c8[3] = __fmul_rn(r0.w, d.y);
+        c8[4] = __fmul_rn(r1.x, d.y); c8[5] = __fmul_rn(r1.y, d.y); c8[6] = __fmul_rn(r1.z, d.y); c8[7] = __fmul_rn(r1.w, d.y);
     }
 
-    const __half *xcol = p.x + kc * 16;
-    int8_t *qcol = p.q + kc * 16;
+    const long long x_img = static_cast<long long>(p.T) * p.K;          // elements per image of x
+    const long long q_img = static_cast<long long>(p.T) * p.q_pitch;    // bytes per image of q
+    const __half *xp = p.x + b * x_img + static_cast<long long>(t) * p.K + kc * 8;
+    int8_t *qp = p.q + b * q_img + static_cast<long long>(t) * p.q_pitch + kc * 8;
+    const long long x_step = S * x_img, q_step = S * q_img;
 
-    // Two rows per trip so that four 16-byte loads are in flight per thread.
-    while (row < p.M) {
-        const long long row2 = row + p.rows_per_iter;
-        int t2 = t + t_step;
-        if (t2 >= p.T) t2 -= p.T;
-        const bool has2 = row2 < p.M;
-
-        const uint4 *src = reinterpret_cast<const uint4 *>(xcol + row * p.K);
-        const uint4 a0 = __ldcs(src), a1 = __ldcs(src + 1);
-        uint4 b0 = make_uint4(0, 0, 0, 0), b1 = b0;
-        if (has2) {
-            const uint4 *src2 = reinterpret_cast<const uint4 *>(xcol + row2 * p.K);
-            b0 = __ldcs(src2);
-            b1 = __ldcs(src2 + 1);
+    uint4 cur[U], nxt[U];
+    auto load_trip = [&](int b0, const __half *src, uint4 (&v)[U]) {
+#pragma unroll
+        for (int j = 0; j < U; ++j) {
+            v[j] = make_uint4(0, 0, 0, 0);
+            if (b0 + j * S < p.B) v[j] = __ldcs(reinterpret_cast<const uint4 *>(src + j * x_step));
         }
-        const float dxa = __ldg(p.dx + t), rdxa = __ldg(p.rdx + t);
-        const float dxb = __ldg(p.dx + t2), rdxb = __ldg(p.rdx + t2);
-
-        uint4 out;
-        quantize8<kFast>(a0.x, a0.y, a0.z, a0.w, s16, rs16, dxa, rdxa, out.x, out.y);
-        quantize8<kFast>(a1.x, a1.y, a1.z, a1.w, s16 + 8, rs16 + 8, dxa, rdxa, out.z, out.w);
-        *reinterpret_cast<uint4 *>(qcol + row * p.q_pitch) = out;
-        if (has2) {
-            quantize8<kFast>(b0.x, b0.y, b0.z, b0.w, s16, rs16, dxb, rdxb, out.x, out.y);
-            quantize8<kFast>(b1.x, b1.y, b1.z, b1.w, s16 + 8, rs16 + 8, dxb, rdxb, out.z, out.w);
-            *reinterpret_cast<uint4 *>(qcol + row2 * p.q_pitch) = out;
+    };
+    load_trip(b, xp, cur);
+    while (b < p.B) {
+        load_trip(b + U * S, xp + U * x_step, nxt);
+#pragma unroll
+        for (int j = 0; j < U; ++j) {
+            if (b + j * S < p.B) {
+                uint2 out;
+                bool exact = !kFast;
+                if (kFast) exact = quantize8_screen(cur[j].x, cur[j].y, cur[j].z, cur[j].w, c8, out.x, out.y);
+                if (exact) quantize8_exact<kFast>(cur[j].x, cur[j].y, cur[j].z, cur[j].w, s8, rs8, d.x, d.y, out.x, out.y);
+                *reinterpret_cast<uint2 *>(qp + j * q_step) = out;
+            }
         }
-        row = row2 + p.rows_per_iter;
-        t = t2 + t_step;
-        if (t >= p.T) t -= p.T;
+#pragma unroll
+        for (int j = 0; j < U; ++j) cur[j] = nxt[j];
+        b += U * S;
+        xp += U * x_step;
+        qp += U * q_step;
     }
 }
 

@@ -41,35 +41,39 @@ def layer_inputs(spec, B=None):
     return x, wq, dw, bias, s, dx
 
 
-def check_layer(ptq, torch, spec, B=None, flags=0, full=None, seed=0):
-    """Forward with taps through the C ABI; compare codes and accumulators bit for bit and the fp16
+def check_layer(ptq, torch, spec, B=None, flags_list=(0, 1), full=None, seed=0):
+    """Forward with taps through the C ABI, once per entry of flags_list (0 = quantize kernel then
+    GEMM kernel, 1 = PTQ_FLAG_FUSED_PROLOGUE); compare codes and accumulators bit for bit and the fp16
     output within tolerance, on every row (small layers) or on sampled row blocks (large ones)."""
     x, wq, dw, bias, s, dx = layer_inputs(spec, B)
     Bn = x.shape[0]
     M = Bn * spec.T
     layer = ptq.PtqLinear(wq, dw, s, dx, bias)
     xd = torch.from_numpy(x).cuda()
-    y, q, acc = layer.forward_debug(xd, flags=flags)
-    y2 = layer.forward(xd, flags=flags)                       # the production entry point
-    torch.cuda.synchronize()
-    layer.device_status()
-    assert torch.equal(y, y2), "forward and forward_debug disagree"
-    y = y.cpu().numpy().reshape(M, spec.N)
-    q = q.cpu().numpy().reshape(M, spec.K)
-    acc = acc.cpu().numpy().reshape(M, spec.N)
     x2 = x.reshape(M, spec.K)
     if full is None:
         full = M * spec.K * spec.N <= 4e9
     blocks = [(0, M)] if full else sample_row_blocks(M, np.random.default_rng(seed))
+    refs = [oracle.linear_forward(x2, spec.T, wq, dw, s, dx, bias, rows=blk, taps=True) for blk in blocks]
+    q_all = None if full else oracle.quantize(x2, spec.T, s, dx)
     clip = 0
-    for (m0, m1) in blocks:
-        y_ref, q_ref, acc_ref = oracle.linear_forward(x2, spec.T, wq, dw, s, dx, bias, rows=(m0, m1), taps=True)
-        assert np.array_equal(q[m0:m1], q_ref), "%s rows %d:%d: int8 codes differ" % (spec.name, m0, m1)
-        assert np.array_equal(acc[m0:m1], acc_ref), "%s rows %d:%d: int32 accumulators differ" % (spec.name, m0, m1)
-        assert_y_close(y[m0:m1], y_ref, "%s rows %d:%d" % (spec.name, m0, m1))
-        clip += int((np.abs(q_ref.astype(np.int32)) >= 127).sum())
-    if not full:
-        # codes are cheap for the oracle: compare all of them even when the matmul is sampled
-        assert np.array_equal(q, oracle.quantize(x2, spec.T, s, dx)), "%s: int8 codes differ" % spec.name
+    for flags in flags_list:
+        what = "%s flags=%d" % (spec.name, flags)
+        y, q, acc = layer.forward_debug(xd, flags=flags)
+        y2 = layer.forward(xd, flags=flags)                   # the production entry point
+        torch.cuda.synchronize()
+        layer.device_status()
+        assert torch.equal(y, y2), "%s: forward and forward_debug disagree" % what
+        y = y.cpu().numpy().reshape(M, spec.N)
+        q = q.cpu().numpy().reshape(M, spec.K)
+        acc = acc.cpu().numpy().reshape(M, spec.N)
+        for (m0, m1), (y_ref, q_ref, acc_ref) in zip(blocks, refs):
+            assert np.array_equal(q[m0:m1], q_ref), "%s rows %d:%d: int8 codes differ" % (what, m0, m1)
+            assert np.array_equal(acc[m0:m1], acc_ref), "%s rows %d:%d: int32 accumulators differ" % (what, m0, m1)
+            assert_y_close(y[m0:m1], y_ref, "%s rows %d:%d" % (what, m0, m1))
+            clip += int((np.abs(q_ref.astype(np.int32)) >= 127).sum())
+        if not full:
+            # codes are cheap for the oracle: compare all of them even when the matmul is sampled
+            assert np.array_equal(q, q_all), "%s: int8 codes differ" % what
     layer.close()
     return clip

@@ -120,6 +120,28 @@ def test_odd_shapes_and_ragged_tiles(env, K, N, T, B):
     check_layer(ptq, torch, spec, full=True)
 
 
+def test_fused_flag_is_reported_and_needs_no_workspace(env):
+    ptq, torch = env
+    for spec, want in ((CFG[3][0], True), (CFG[3][1], True), (CFG[1][2], False),
+                       (wl.LinearSpec(9, 0, 0, "bigk", 2, 5, 4096, 64), False)):
+        x, wq, dw, bias, s, dx = layer_inputs(spec, B=2)
+        layer = ptq.PtqLinear(wq, dw, s, dx, bias)
+        assert layer.fused_supported() == want
+        if want:
+            assert layer.workspace_bytes(2, ptq.FLAG_FUSED_PROLOGUE) == 0
+            xd = torch.from_numpy(x).cuda()
+            y = torch.empty((2, spec.T, spec.N), dtype=torch.float16, device="cuda")
+            L = ptq.load_library()
+            st = L.ptq_linear_forward(layer._h, xd.data_ptr(), 2, y.data_ptr(), None, 0, ptq.FLAG_FUSED_PROLOGUE, None)
+            assert st == 0
+            torch.cuda.synchronize()
+            layer.device_status()
+            y_ref = oracle.linear_forward(x.reshape(-1, spec.K), spec.T, wq, dw, s, dx, bias)
+            assert_y_close(y.cpu().numpy().reshape(-1, spec.N), y_ref, "fused without workspace")
+        else:
+            assert layer.workspace_bytes(2, ptq.FLAG_FUSED_PROLOGUE) == layer.workspace_bytes(2, 0) > 0
+
+
 def test_unaligned_pointers_take_the_generic_paths(env):
     ptq, torch = env
     spec = CFG[0][0]
@@ -131,11 +153,14 @@ def test_unaligned_pointers_take_the_generic_paths(env):
     xv = xbuf[1:1 + x.size].view(2, spec.T, spec.K)          # 2-byte aligned only
     yv = ybuf[1:1 + M * spec.N].view(2, spec.T, spec.N)
     xv.copy_(torch.from_numpy(x).cuda())
-    layer.forward(xv, y=yv)
-    torch.cuda.synchronize()
-    layer.device_status()
     y_ref = oracle.linear_forward(x.reshape(M, spec.K), spec.T, wq, dw, s, dx, bias)
-    assert_y_close(yv.cpu().numpy().reshape(M, spec.N), y_ref, "unaligned")
+    for flags in (0, ptq.FLAG_FUSED_PROLOGUE):       # the fused flag falls back: x is not 16-byte aligned
+        yv.zero_()
+        layer.forward(xv, y=yv, workspace=torch.empty(layer.workspace_bytes(2), dtype=torch.uint8, device="cuda"),
+                      flags=flags)
+        torch.cuda.synchronize()
+        layer.device_status()
+        assert_y_close(yv.cpu().numpy().reshape(M, spec.N), y_ref, "unaligned flags=%d" % flags)
     assert float(ybuf[0]) == 0.0 and float(ybuf[-7:].abs().max()) == 0.0     # nothing written outside y
 
 
@@ -151,8 +176,9 @@ def test_repeated_runs_are_bit_identical_and_stay_inside_y(env):
     yv = ybuf[guard:guard + M * spec.N].view(16, spec.T, spec.N)
     ws = torch.empty(layer.workspace_bytes(16) + 2 * guard, dtype=torch.uint8, device="cuda")
     first = None
-    for _ in range(10):
-        layer.forward(xd, y=yv, workspace=ws[guard:guard + layer.workspace_bytes(16)])
+    for i in range(12):
+        layer.forward(xd, y=yv, workspace=ws[guard:guard + layer.workspace_bytes(16)],
+                      flags=ptq.FLAG_FUSED_PROLOGUE if i % 2 else 0)     # both paths give the same bits
         cur = yv.clone()
         first = cur if first is None else first
         assert torch.equal(cur, first)
