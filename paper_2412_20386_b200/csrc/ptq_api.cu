@@ -113,6 +113,8 @@ struct ptq_linear {
     float2 *d_dx2 = nullptr;                             // [T] {dx, 1/dx}
     unsigned *d_status = nullptr;
     CUtensorMap tmW;
+    CUtensorMap tmWh;          // same weights, box of BN/2 rows: the half tile one CTA of a pair loads
+    int max_pairs = 0;         // resident 2-CTA clusters of the pair kernel on this device (0: not available)
     // A-stationary kernel (fused, and the two-kernel path's GEMM when the code panel fits shared memory)
     bool as_ok = false;
     int as_BN = 0, as_n_tiles = 0, as_w_stages = 0, as_w_stage_bytes = 0, as_staging = 0, as_smem = 0;
@@ -143,6 +145,40 @@ ptq_status_t ensure_smem(Kern kern, int bytes)
 {
     PTQ_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
     return PTQ_OK;
+}
+
+// How many 2-CTA clusters of the pair kernel can be resident at once (0 if cluster launch is unavailable).
+int query_max_pairs()
+{
+    static int cached = -1;
+    static std::mutex mu;
+    std::lock_guard<std::mutex> lock(mu);
+    if (cached >= 0) return cached;
+    cached = 0;
+    if (cudaFuncSetAttribute(ptq::ptq_gemm_dequant_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             ptq::kPairSmemBytes) != cudaSuccess ||
+        cudaFuncSetAttribute(ptq::ptq_gemm_dequant_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             ptq::kPairSmemBytes) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return cached;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2, 1, 1);
+    cfg.blockDim = dim3(ptq::kGemmThreads, 1, 1);
+    cfg.dynamicSmemBytes = ptq::kPairSmemBytes;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, ptq::ptq_gemm_dequant_pair_kernel<false>, &cfg) == cudaSuccess && n > 0)
+        cached = n;
+    else
+        (void)cudaGetLastError();
+    return cached;
 }
 
 // Q1 launch: codes to `q` with `q_pitch` bytes between rows.
@@ -249,6 +285,30 @@ ptq_status_t launch_gemm(const ptq_linear *h, const void *codes, long long M, vo
     p.y_vec2 = (h->N % 2 == 0 && reinterpret_cast<uintptr_t>(y) % 4 == 0) ? 1 : 0;
     p.y_vec8 = 0;   // this kernel always has a staging buffer; 16-byte alignment means TMA stores
 
+    const long long pair_tiles = static_cast<long long>((p.m_tiles + 1) / 2) * p.n_tiles;
+    if (h->max_pairs > 0 && pair_tiles >= h->max_pairs) {
+        // enough 256-row tiles to occupy every CTA pair: cta_group::2 kernel (half the weight bytes per CTA)
+        const int npairs = h->max_pairs;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(2 * npairs, 1, 1);
+        cfg.blockDim = dim3(ptq::kGemmThreads, 1, 1);
+        cfg.dynamicSmemBytes = ptq::kPairSmemBytes;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        if (acc_out)
+            PTQ_CUDA(cudaLaunchKernelEx(&cfg, ptq::ptq_gemm_dequant_pair_kernel<true>, tmA, h->tmWh, tmY, p));
+        else
+            PTQ_CUDA(cudaLaunchKernelEx(&cfg, ptq::ptq_gemm_dequant_pair_kernel<false>, tmA, h->tmWh, tmY, p));
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+        PTQ_CUDA(cudaGetLastError());
+        return PTQ_OK;
+    }
     const long long tiles = static_cast<long long>(p.m_tiles) * p.n_tiles;
     const int grid = static_cast<int>(tiles < h->num_sms ? tiles : h->num_sms);
     if (acc_out)
@@ -366,11 +426,11 @@ ptq_status_t launch_astat(const ptq_linear *h, const void *src, bool quantize, l
                : launch_astat_kernel(ptq::ptq_fused_linear_kernel<false, true, false>, th, h, tmA, tmY, fp, grid, stream);
 }
 
-// G1 + E1 on codes: the A-stationary kernel when the layer's code panel fits, else the streaming one.
+// G1 + E1 on codes.  The streaming kernels keep more bytes in flight from L2 than the A-stationary one
+// (whose resident code panel leaves little shared memory for weight stages) and measure faster.
 ptq_status_t launch_gemm_any(const ptq_linear *h, const void *codes, long long M, void *y, void *acc_out,
                              cudaStream_t stream)
 {
-    if (h->as_ok) return launch_astat(h, codes, false, M, y, acc_out, stream);
     return launch_gemm(h, codes, M, y, acc_out, stream);
 }
 
@@ -542,6 +602,11 @@ ptq_status_t ptq_linear_create(ptq_linear_t **out, int K, int N, int T, const in
                          static_cast<unsigned long long>(Npad), static_cast<unsigned long long>(h->Kpad), ptq::kBK,
                          static_cast<unsigned>(h->BN));
         if (st != PTQ_OK) break;
+        st = make_map_2d(&h->tmWh, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, h->d_w, static_cast<unsigned long long>(K),
+                         static_cast<unsigned long long>(Npad), static_cast<unsigned long long>(h->Kpad), ptq::kBK,
+                         static_cast<unsigned>(h->BN / 2));
+        if (st != PTQ_OK) break;
+        h->max_pairs = query_max_pairs();
         if (h->as_ok)
             st = make_map_2d(&h->tmWas, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, h->d_w, static_cast<unsigned long long>(K),
                              static_cast<unsigned long long>(Npad), static_cast<unsigned long long>(h->Kpad),

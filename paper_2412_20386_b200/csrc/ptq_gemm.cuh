@@ -355,4 +355,189 @@ ptq_gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     }
 }
 
+// --- CTA-pair variant --------------------------------------------------------------------------
+//
+// Same computation with tcgen05 cta_group::2: two CTAs (a cluster of 2 on neighbouring SMs) share one
+// 256 x BN output tile.  Each CTA loads its own 128 rows of codes and only HALF of the weight tile
+// (BN/2 rows); the leader CTA issues one MMA that reads both CTAs' shared memory and writes 128
+// accumulator rows into each CTA's TMEM.  Per CTA and k-block that is 16 KB + 8..16 KB from L2 instead
+// of 16 KB + 16..32 KB, which is what the 128 x 256 single-CTA tile is short of: its main loop waits
+// on L2, not on the tensor core.  No load is multicast: every CTA fetches only what it stores.
+//
+// Barrier protocol (all barriers live at the same offsets in both CTAs):
+//   full[s]    leader's copy only: one arrive.expect_tx by the leader's producer for the bytes of BOTH
+//              CTAs; every TMA load of either CTA credits the leader's barrier
+//   empty[s]   both copies, signalled together by the leader's multicast tcgen05.commit
+//   tfull[b]   both copies, multicast commit; each CTA's epilogue drains its own TMEM
+//   tempty[b]  leader's copy only, count = epilogue warps of both CTAs (remote arrive from the peer)
+constexpr int kPairStages = 6;
+constexpr int kPairBHalfBytes = (kMaxBN / 2) * kBK;                   // 16 KB
+constexpr int kPairStageBytes = kATileBytes + kPairBHalfBytes;         // 32 KB
+constexpr int kPairNumBarriers = 2 * kPairStages + 4;
+constexpr int kPairSmemBytes =
+    1024 + kPairStages * kPairStageBytes + kNumEpiWarps * kStagingBytesPerWarp + kPairNumBarriers * 8 + 16;
+
+template <bool kDebugAcc>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+ptq_gemm_dequant_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmWh,
+                             const __grid_constant__ CUtensorMap tmY, const GemmParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t *base_ptr = smem_raw + (base - raw);
+    const uint32_t staging_base = base + kPairStages * kPairStageBytes;
+    const uint32_t bar_off = kPairStages * kPairStageBytes + kNumEpiWarps * kStagingBytesPerWarp;
+    const uint32_t bar_base = base + bar_off;
+    auto full_bar = [&](uint32_t s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](uint32_t s) { return bar_base + 8u * (kPairStages + s); };
+    auto tfull_bar = [&](uint32_t b) { return bar_base + 8u * (2 * kPairStages + b); };
+    auto tempty_bar = [&](uint32_t b) { return bar_base + 8u * (2 * kPairStages + 2 + b); };
+    volatile uint32_t *tmem_holder = reinterpret_cast<volatile uint32_t *>(base_ptr + bar_off + kPairNumBarriers * 8);
+    volatile uint32_t *abort_flag = tmem_holder + 1;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_cta_rank();          // 0 = leader
+    const int pair = blockIdx.x >> 1;
+    const int npairs = gridDim.x >> 1;
+    const int half_bn = p.BN >> 1;                       // weight rows per CTA
+
+    if (threadIdx.x == 0) {
+        for (uint32_t s = 0; s < kPairStages; ++s) {
+            mbar_init(full_bar(s), 1);
+            mbar_init(empty_bar(s), 1);
+        }
+        for (uint32_t b = 0; b < 2; ++b) {
+            mbar_init(tfull_bar(b), 1);
+            mbar_init(tempty_bar(b), 2 * kNumEpiWarps);
+        }
+        *abort_flag = 0u;
+        fence_mbar_init();
+        prefetch_tensormap(&tmA);
+        prefetch_tensormap(&tmWh);
+        if (p.use_tma_store) prefetch_tensormap(&tmY);
+    }
+    if (warp == 1) {
+        tmem_alloc_pair(smem_u32(const_cast<uint32_t *>(tmem_holder)), kTmemCols);
+        tmem_relinquish_alloc_permit_pair();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    cluster_sync_all();                                  // both CTAs' barriers exist before anyone signals them
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_holder;
+
+    const int pair_m_tiles = (p.m_tiles + 1) >> 1;       // 256-row tiles
+    const int total_tiles = pair_m_tiles * p.n_tiles;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer (both CTAs)
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0, issued = 0;
+            bool ok = true;
+            const uint32_t stage_tx = 2u * static_cast<uint32_t>(kATileBytes + half_bn * kBK);
+            for (int tile = pair; tile < total_tiles && ok; tile += npairs) {
+                const int m_tile = tile / p.n_tiles;
+                const int n_tile = tile - m_tile * p.n_tiles;
+                for (int kb = 0; kb < p.k_blocks; ++kb) {
+                    if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status)) {
+                        ok = false;
+                        break;
+                    }
+                    const uint32_t a_dst = base + stage * kPairStageBytes;
+                    if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), stage_tx);
+                    tma_load_2d_pair(a_dst, &tmA, kb * kBK, m_tile * (2 * kBM) + static_cast<int>(rank) * kBM,
+                                     full_bar(stage));
+                    tma_load_2d_pair(a_dst + kATileBytes, &tmWh, kb * kBK,
+                                     n_tile * p.BN + static_cast<int>(rank) * half_bn, full_bar(stage));
+                    ++issued;
+                    if (++stage == kPairStages) {
+                        stage = 0;
+                        phase ^= 1u;
+                    }
+                }
+            }
+            if (!ok && rank == 0) {
+                // Error path only: let the loads already issued land (bounded).
+                for (uint32_t s = 0; s < kPairStages; ++s) {
+                    const uint32_t uses = (issued + kPairStages - 1u - s) / kPairStages;
+                    if (uses == 0u) continue;
+                    for (int i = 0; i < 200000 && !mbar_try_wait(full_bar(s), (uses - 1u) & 1u); ++i) {
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer (leader only)
+        if (lane == 0 && rank == 0) {
+            const uint32_t idesc = make_idesc_s8(2 * kBM, p.BN);
+            uint32_t stage = 0, phase = 0, buf = 0, bphase = 0;
+            bool ok = true;
+            for (int tile = pair; tile < total_tiles && ok; tile += npairs) {
+                if (!mbar_wait(tempty_bar(buf), bphase ^ 1u, abort_flag, p.status)) break;
+                tc_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + buf * kMaxBN;
+                for (int kb = 0; kb < p.k_blocks; ++kb) {
+                    if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after_sync();
+                    const uint32_t a_addr = base + stage * kPairStageBytes;
+                    const uint64_t a_desc = make_smem_desc_sw128(a_addr);
+                    const uint64_t b_desc = make_smem_desc_sw128(a_addr + kATileBytes);
+                    const int nmma = (kb == p.k_blocks - 1) ? p.last_mmas : (kBK / 32);
+                    for (int j = 0; j < nmma; ++j)
+                        mma_i8_ss_pair(d_tmem, a_desc + 2u * j, b_desc + 2u * j, idesc, (kb | j) != 0 ? 1u : 0u);
+                    mma_commit_pair(empty_bar(stage));
+                    if (++stage == kPairStages) {
+                        stage = 0;
+                        phase ^= 1u;
+                    }
+                }
+                if (!ok) break;
+                mma_commit_pair(tfull_bar(buf));
+                buf ^= 1u;
+                if (buf == 0u) bphase ^= 1u;
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue warps (both CTAs)
+        const int quarter = warp & 3;
+        const int col_half = (warp - 2) >> 2;
+        const uint32_t staging = staging_base + static_cast<uint32_t>(warp - 2) * kStagingBytesPerWarp;
+        uint32_t buf = 0, bphase = 0, nboxes = 0;
+        for (int tile = pair; tile < total_tiles; tile += npairs) {
+            const int m_tile = tile / p.n_tiles;
+            const int n_tile = tile - m_tile * p.n_tiles;
+            const long long m_row0 =
+                static_cast<long long>(m_tile) * (2 * kBM) + static_cast<long long>(rank) * kBM + quarter * 32;
+            const long long m = m_row0 + lane;
+            const float dxr = (m < p.M) ? __ldg(p.dx + static_cast<int>(m % p.T)) : 0.0f;
+            bool got = mbar_wait(tfull_bar(buf), bphase, abort_flag, p.status);
+            got = __all_sync(0xffffffffu, got);
+            if (!got) break;
+            tc_fence_after_sync();
+            const uint32_t tmem_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * kMaxBN;
+            nboxes = epilogue_tile<kDebugAcc>(p, &tmY, tmem_row, m_row0, n_tile * p.BN, dxr, staging, nboxes, lane,
+                                              col_half);
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_remote(tempty_bar(buf), 0u);     // the leader's MMA thread waits on it
+            buf ^= 1u;
+            if (buf == 0u) bphase ^= 1u;
+        }
+        if (lane == 0) bulk_wait_group<0>();
+    }
+
+    __syncthreads();
+    cluster_sync_all();          // the peer may still signal this CTA's barriers or be read by the leader's MMAs
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after_sync();
+        tmem_dealloc_pair(tmem_base, kTmemCols);
+    }
+}
+
 }  // namespace ptq
