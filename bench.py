@@ -76,7 +76,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
-                 "--format=csv,noheader,nounits", "-lms", "100"],
+                 "--format=csv,noheader,nounits", "-lms", "50"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
@@ -86,9 +86,11 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.lines.append(line.strip())
+            self.lines.append((time.time(), line.strip()))
 
-    def stop(self):
+    def stop(self, t0=None, t1=None, t2=None):
+        """Summarise the samples taken in [t0, t1] (the timed region); if fewer than three fall inside
+        it, widen to [t0, t2] (the end-to-end loop that follows, same kernels) and say so."""
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         self.proc.terminate()
@@ -96,9 +98,14 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
+        window = "timed region"
+        lines = [l for (ts, l) in self.lines if t0 is None or (t0 <= ts <= t1)]
+        if t0 is not None and len(lines) < 3:
+            lines = [l for (ts, l) in self.lines if t0 <= ts <= (t2 or t1)]
+            window = "timed region + end-to-end loop"
         sm, smax, reasons = [], [], set()
         names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
-        for line in self.lines:
+        for line in lines:
             parts = [p.strip() for p in line.split(",")]
             if len(parts) < 6:
                 continue
@@ -112,7 +119,7 @@ class ClockSampler:
                     reasons.add(n)
         return {"sm_mhz": statistics.median(sm) if sm else None,
                 "sm_max_mhz": max(smax) if smax else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+                "reasons": sorted(reasons), "samples": len(sm), "window": window}
 
 
 # ------------------------------------------------------------------------------------------------
@@ -129,60 +136,72 @@ def oracle_layer_inputs(spec, rows):
     return x, wq, dw, bias, s, dx
 
 
-def time_oracle(specs, target_seconds, repeats=1):
-    """Times the oracle's whole path on the leading rows of every layer; the row count is sized by a
-    short probe so that one pass takes about `target_seconds`.  Returns (TOPS, sample text, seconds)."""
+def plan_oracle(specs, target_seconds):
+    """Sizes a row sample per layer (leading rows, whole images generated) so that one pass of the
+    oracle over all layers takes about `target_seconds`; a short probe per layer gives its rate."""
     import oracle
     total_ops_full = sum(layer_ops(sp, sp.B) for sp in specs)
-    plans = []
+    data = []
     for sp in specs:
-        probe_rows = min(sp.M, 256)
+        probe_rows = min(sp.M, 128)
         x, wq, dw, bias, s, dx = oracle_layer_inputs(sp, probe_rows)
         t0 = time.perf_counter()
         oracle.linear_forward(x, sp.T, wq, dw, s, dx, bias, rows=(0, probe_rows))
         dt = max(time.perf_counter() - t0, 1e-6)
         share = layer_ops(sp, sp.B) / total_ops_full
-        rows = int(min(sp.M, max(probe_rows, probe_rows * (target_seconds * share) / dt)))
-        plans.append((sp, rows))
+        rows = int(min(sp.M, max(8, probe_rows * (target_seconds * share) / dt)))
+        if rows > x.shape[0]:
+            x, wq, dw, bias, s, dx = oracle_layer_inputs(sp, rows)
+        data.append((sp, rows, (x, wq, dw, bias, s, dx)))
+    sample = "; ".join("c%d L%d %s: first %d of %d rows" % (sp.config, sp.layer, sp.name, rows, sp.M)
+                       for sp, rows, _ in data[:6])
+    if len(data) > 6:
+        sample += "; ... (%d layers)" % len(data)
+    return data, sample
+
+
+def run_oracle_pass(data):
+    """One pass of the oracle's whole path over the planned samples: (ops, seconds)."""
+    import oracle
     ops = 0.0
     secs = 0.0
-    data = [(sp, rows, oracle_layer_inputs(sp, rows)) for sp, rows in plans]
-    for _ in range(repeats):
-        for sp, rows, (x, wq, dw, bias, s, dx) in data:
-            rows = min(rows, x.shape[0])
-            t0 = time.perf_counter()
-            oracle.linear_forward(x, sp.T, wq, dw, s, dx, bias, rows=(0, rows))
-            secs += time.perf_counter() - t0
-            ops += 2.0 * rows * sp.K * sp.N
-    sample = "; ".join("%s L%d %s: first %d of %d rows" % ("c%d" % sp.config, sp.layer, sp.name, rows, sp.M)
-                       for sp, rows in plans[:6])
-    if len(plans) > 6:
-        sample += "; ... (%d layers)" % len(plans)
+    for sp, rows, (x, wq, dw, bias, s, dx) in data:
+        t0 = time.perf_counter()
+        oracle.linear_forward(x, sp.T, wq, dw, s, dx, bias, rows=(0, rows))
+        secs += time.perf_counter() - t0
+        ops += 2.0 * rows * sp.K * sp.N
+    return ops, secs
+
+
+def time_oracle(specs, target_seconds):
+    """(TOPS, sample text, seconds) of one oracle pass sized to about `target_seconds`."""
+    data, sample = plan_oracle(specs, target_seconds)
+    ops, secs = run_oracle_pass(data)
     return ops / secs / 1e12, sample, secs
 
 
 def run_reference(args, specs, rank):
+    """The reference arm: the CPU oracle, as it stands, on the host cores.  Each step is one pass over
+    a bounded row sample of the workload, sized so that warm-up plus steps stay within ~2.5 minutes."""
     if rank != 0:
         return
     import oracle
-    per_step = 2.0
-    t_all = time.perf_counter()
+    per_step = min(2.0, max(0.01, 150.0 / max(1, args.steps + args.warmup)))
+    data, sample = plan_oracle(specs, per_step)
     for _ in range(args.warmup):
-        time_oracle(specs, per_step * 0.25)
-    vals = []
-    sample = ""
+        run_oracle_pass(data)
+    ops = secs = 0.0
     for _ in range(args.steps):
-        v, sample, _ = time_oracle(specs, per_step)
-        vals.append(v)
-    # whole-run throughput = total ops / total time = harmonic-style mean over equal-length steps
-    value = len(vals) / sum(1.0 / v for v in vals)
+        o, t = run_oracle_pass(data)
+        ops += o
+        secs += t
+    value = ops / secs / 1e12
     cores = oracle.num_threads()
     out = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": 1e3 * (time.perf_counter() - t_all) / max(1, args.steps + args.warmup),
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * secs / max(1, args.steps),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
-        "config": {"workload": args.workload, "layers": len(specs)},
+        "config": {"workload": args.workload, "n_layers": len(specs), "path": "cpu oracle"},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -193,6 +212,23 @@ def run_reference(args, specs, rank):
 # ------------------------------------------------------------------------------------------------
 # GPU arm
 # ------------------------------------------------------------------------------------------------
+def reduce_max_over_ranks(values, device=None):
+    """Element-wise maximum of a list of floats over all ranks of the default process group (the job's
+    time is the slowest rank's); the identity without a process group."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return [float(v) for v in values]
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def whole_job_tops(world, step_ops_per_rank, ms_per_step):
+    """Replicas: every rank does step_ops_per_rank in the (max over ranks) step time."""
+    return world * step_ops_per_rank / (ms_per_step * 1e-3) / 1e12
+
+
 def event_times_ms(torch, fn, iters):
     """Average device time of fn() per call, each call bracketed by its own CUDA events on the
     current stream (the stream the library launches on)."""
@@ -222,7 +258,7 @@ def run_ours(args, specs, rank, world, local_rank):
     dev = torch.device("cuda", local_rank)
     peaks, peaks_kind = load_peaks()
 
-    flags = ptq.FLAG_FUSED_PROLOGUE if args.path == "fused" else 0
+    flags = {"unfused": 0, "fused": ptq.FLAG_FUSED_PROLOGUE, "pair": ptq.FLAG_CTA_PAIR}[args.path]
     layers = []
     for sp in specs:
         x_host = torch.from_numpy(wl.activations(sp, wl.ROLE_EVAL)).pin_memory()
@@ -236,7 +272,7 @@ def run_ours(args, specs, rank, world, local_rank):
         ws_bytes = layer.workspace_bytes(sp.B, flags)
         ws = torch.empty(max(ws_bytes, 16), dtype=torch.uint8, device=dev)
         layers.append(dict(spec=sp, layer=layer, x_host=x_host, x=x_dev, y=y_dev, y_host=y_host, ws=ws,
-                           fused=bool(flags and layer.fused_supported())))
+                           fused=bool((flags & ptq.FLAG_FUSED_PROLOGUE) and layer.fused_supported())))
     step_ops = sum(layer_ops(d["spec"], d["spec"].B) for d in layers)
     touched = sum(d["x"].numel() * 2 + d["y"].numel() * 2 for d in layers)
 
@@ -265,14 +301,15 @@ def run_ours(args, specs, rank, world, local_rank):
     n0 = ptq.binding.kernel_launch_count()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
+    t_start = time.time()
     e0.record()
     for _ in range(args.steps):
         step()
     e1.record()
     barrier()
+    t_end = time.time()
     launches = ptq.binding.kernel_launch_count() - n0
     ms_total = e0.elapsed_time(e1)
-    clocks = sampler.stop()
     for d in layers:
         d["layer"].device_status()
 
@@ -288,15 +325,12 @@ def run_ours(args, specs, rank, world, local_rank):
     f1.record()
     barrier()
     ms_e2e = f0.elapsed_time(f1) / e2e_steps
+    clocks = sampler.stop(t_start, t_end, time.time())
 
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total, ms_e2e = float(t[0]), float(t[1])
+    ms_total, ms_e2e = reduce_max_over_ranks([ms_total, ms_e2e], dev)
     ms_step = ms_total / args.steps
-    value = world * step_ops / (ms_step * 1e-3) / 1e12
-    e2e_value = world * step_ops / (ms_e2e * 1e-3) / 1e12
+    value = whole_job_tops(world, step_ops, ms_step)
+    e2e_value = whole_job_tops(world, step_ops, ms_e2e)
 
     if rank != 0:
         return
@@ -305,7 +339,7 @@ def run_ours(args, specs, rank, world, local_rank):
     int8_peak = peaks["bf16_tflops_sustained"] * INT8_OVER_BF16
     hbm_peak = peaks["hbm_gbs"]
     kernels = []
-    iters = max(10, min(args.steps, 50))
+    iters = 50
     for d in layers:
         sp, layer = d["spec"], d["layer"]
         M, K, N = sp.M, sp.K, sp.N
@@ -321,7 +355,11 @@ def run_ours(args, specs, rank, world, local_rank):
             avg, mn, med = event_times_ms(torch, lambda: layer.quantize(d["x"], q=qdense), iters)
             kernels.append(dict(kernel="ptq_quantize_kernel", layer=tag, ms=avg, ms_min=mn, ops=0.0, bytes=3.0 * M * K))
             layer.forward(d["x"], y=d["y"], workspace=d["ws"], flags=0)      # leaves valid codes in ws
-            avg, mn, med = event_times_ms(torch, lambda: layer.gemm_dequant(codes, sp.B, y=d["y"]), iters)
+            if flags & ptq.FLAG_CTA_PAIR:                                    # time the pair GEMM as forward minus quantize
+                tot, _, _ = event_times_ms(torch, lambda: layer.forward(d["x"], y=d["y"], workspace=d["ws"], flags=flags), iters)
+                avg, mn = max(tot - avg, 1e-6), max(tot - avg, 1e-6)
+            else:
+                avg, mn, med = event_times_ms(torch, lambda: layer.gemm_dequant(codes, sp.B, y=d["y"]), iters)
             kernels.append(dict(kernel="ptq_gemm_dequant_kernel", layer=tag, ms=avg, ms_min=mn, ops=2.0 * M * K * N,
                                 bytes=1.0 * M * K + N * K + 2.0 * M * N))
             del qdense
@@ -389,11 +427,13 @@ TRAFFIC = {}
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c3", choices=["c0", "c1", "c2", "c3", "c4"])
-    ap.add_argument("--path", default="unfused", choices=["unfused", "fused"])
+    ap.add_argument("--path", default="unfused", choices=["unfused", "fused", "pair"],
+                    help="unfused: quantize kernel + GEMM kernel (fastest at present, the default); "
+                         "fused: PTQ_FLAG_FUSED_PROLOGUE; pair: PTQ_FLAG_CTA_PAIR")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup

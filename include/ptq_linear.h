@@ -59,6 +59,8 @@ typedef enum {
 /* Flags for create / forward. */
 #define PTQ_FLAG_NONE            0u
 #define PTQ_FLAG_FUSED_PROLOGUE  1u   /* F1: quantize inside the GEMM kernel; no int8 round trip, no workspace */
+#define PTQ_FLAG_CTA_PAIR        2u   /* two-kernel path: run G1+E1 on CTA pairs (tcgen05 cta_group::2, 256-row tiles,
+                                         half the weight bytes per CTA) when the batch has enough rows; same results */
 
 /* Limits (create returns PTQ_ERR_SHAPE beyond them). */
 #define PTQ_MAX_K   8192
@@ -194,6 +196,13 @@ ptq_status_t ptq_calibrate(int K, int N, int T, const void *xcal_fp16, int Bc,
  * call (its output is then undefined), or PTQ_ERR_CUDA.
  */
 ptq_status_t ptq_linear_device_status(const ptq_linear_t *h);
+
+/*
+ * Write a one-line, human-readable description of the kernels and tilings chosen for this layer
+ * (tile sizes, stage counts, whether PTQ_FLAG_FUSED_PROLOGUE has a kernel for it) into buf (at most
+ * buf_bytes including the terminating NUL).  Returns the length the full text needs.
+ */
+int ptq_linear_describe(const ptq_linear_t *h, char *buf, int buf_bytes);
 
 /* Number of kernels this library has launched in the calling process (all handles, all threads). */
 unsigned long long ptq_kernel_launch_count(void);

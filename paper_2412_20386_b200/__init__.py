@@ -8,4 +8,4 @@ and the binding raises if it is missing: there is no CPU fallback.
 """
 from . import workloads  # noqa: F401
 from .binding import (PtqError, PtqLinear, calibrate, library_path, load_library,  # noqa: F401
-                      FLAG_FUSED_PROLOGUE)
+                      FLAG_FUSED_PROLOGUE, FLAG_CTA_PAIR)

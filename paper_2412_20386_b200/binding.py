@@ -19,6 +19,7 @@ _SO = os.path.join(_HERE, "libptq_linear.so")
 
 FLAG_NONE = 0
 FLAG_FUSED_PROLOGUE = 1
+FLAG_CTA_PAIR = 2
 STATIC_SCRATCH_BYTES = 32 * 1024 * 1024
 
 _STATUS_NAMES = {0: "PTQ_OK", 1: "PTQ_ERR_NULL", 2: "PTQ_ERR_SHAPE", 3: "PTQ_ERR_VALUE",
@@ -71,6 +72,8 @@ def load_library() -> ctypes.CDLL:
     L.ptq_linear_forward_debug.argtypes = [vp, vp, ci, vp, vp, vp, vp, sz, cu, vp]
     L.ptq_calibrate.restype = ci
     L.ptq_calibrate.argtypes = [ci, ci, ci, vp, ci, vp, vp, vp, vp, vp]
+    L.ptq_linear_describe.restype = ci
+    L.ptq_linear_describe.argtypes = [vp, ctypes.c_char_p, ci]
     L.ptq_linear_device_status.restype = ci
     L.ptq_linear_device_status.argtypes = [vp]
     L.ptq_kernel_launch_count.restype = ctypes.c_ulonglong
@@ -149,6 +152,11 @@ class PtqLinear:
 
     def fused_supported(self) -> bool:
         return bool(self._L.ptq_linear_fused_supported(self._h))
+
+    def describe(self) -> str:
+        buf = ctypes.create_string_buffer(512)
+        self._L.ptq_linear_describe(self._h, buf, 512)
+        return buf.value.decode()
 
     def device_status(self):
         _check(self._L.ptq_linear_device_status(self._h))

@@ -240,7 +240,7 @@ ptq_status_t launch_quantize(const ptq_linear *h, const void *x, long long M, vo
 
 // G1+E1 launch on codes [M, Kpad] at `codes`.
 ptq_status_t launch_gemm(const ptq_linear *h, const void *codes, long long M, void *y, void *acc_out,
-                         cudaStream_t stream)
+                         cudaStream_t stream, bool want_pair = false)
 {
     static std::once_flag once;
     static ptq_status_t attr_status = PTQ_OK;
@@ -286,7 +286,7 @@ ptq_status_t launch_gemm(const ptq_linear *h, const void *codes, long long M, vo
     p.y_vec8 = 0;   // this kernel always has a staging buffer; 16-byte alignment means TMA stores
 
     const long long pair_tiles = static_cast<long long>((p.m_tiles + 1) / 2) * p.n_tiles;
-    if (h->max_pairs > 0 && pair_tiles >= h->max_pairs) {
+    if (want_pair && h->max_pairs > 0 && pair_tiles >= h->max_pairs) {
         // enough 256-row tiles to occupy every CTA pair: cta_group::2 kernel (half the weight bytes per CTA)
         const int npairs = h->max_pairs;
         cudaLaunchConfig_t cfg = {};
@@ -429,9 +429,9 @@ ptq_status_t launch_astat(const ptq_linear *h, const void *src, bool quantize, l
 // G1 + E1 on codes.  The streaming kernels keep more bytes in flight from L2 than the A-stationary one
 // (whose resident code panel leaves little shared memory for weight stages) and measure faster.
 ptq_status_t launch_gemm_any(const ptq_linear *h, const void *codes, long long M, void *y, void *acc_out,
-                             cudaStream_t stream)
+                             cudaStream_t stream, bool want_pair = false)
 {
-    return launch_gemm(h, codes, M, y, acc_out, stream);
+    return launch_gemm(h, codes, M, y, acc_out, stream, want_pair);
 }
 
 bool fused_usable(const ptq_linear *h) { return h->as_ok && h->K % 16 == 0; }
@@ -647,6 +647,24 @@ ptq_status_t ptq_quantize(const ptq_linear_t *h, const void *x_fp16, int B, void
     return launch_quantize(h, x_fp16, M, q_int8, h->K, static_cast<cudaStream_t>(stream));
 }
 
+int ptq_linear_describe(const ptq_linear_t *h, char *buf, int buf_bytes)
+{
+    if (!h) return 0;
+    char tmp[512];
+    const int n = snprintf(tmp, sizeof(tmp),
+                           "K=%d N=%d T=%d Kpad=%d | quantize: %s | gemm: BN=%d n_tiles=%d k_blocks=%d "
+                           "pair_clusters=%d | fused: %s BN=%d n_tiles=%d w_stages=%d staging=%d smem=%d",
+                           h->K, h->N, h->T, h->Kpad, h->fast_div ? "screened reciprocal route" : "IEEE division",
+                           h->BN, h->n_tiles, h->k_blocks, h->max_pairs,
+                           (h->as_ok && h->K % 16 == 0) ? "yes" : "no", h->as_BN, h->as_n_tiles, h->as_w_stages,
+                           h->as_staging, h->as_smem);
+    if (buf && buf_bytes > 0) {
+        strncpy(buf, tmp, static_cast<size_t>(buf_bytes) - 1);
+        buf[buf_bytes - 1] = 0;
+    }
+    return n;
+}
+
 int ptq_linear_code_pitch(const ptq_linear_t *h) { return h ? h->Kpad : 0; }
 
 ptq_status_t ptq_linear_gemm_dequant(const ptq_linear_t *h, const void *q_int8, int B, void *y_fp16, void *stream)
@@ -669,7 +687,7 @@ ptq_status_t ptq_linear_forward_debug(const ptq_linear_t *h, const void *x_fp16,
 {
     ptq_status_t st = validate_forward(h, x_fp16, B, y_fp16);
     if (st != PTQ_OK) return st;
-    if (flags & ~PTQ_FLAG_FUSED_PROLOGUE) return fail(PTQ_ERR_VALUE, "unknown flags 0x%x", flags);
+    if (flags & ~(PTQ_FLAG_FUSED_PROLOGUE | PTQ_FLAG_CTA_PAIR)) return fail(PTQ_ERR_VALUE, "unknown flags 0x%x", flags);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const long long M = static_cast<long long>(B) * h->T;
     if ((flags & PTQ_FLAG_FUSED_PROLOGUE) && fused_usable(h) && reinterpret_cast<uintptr_t>(x_fp16) % 16 == 0) {
@@ -688,7 +706,8 @@ ptq_status_t ptq_linear_forward_debug(const ptq_linear_t *h, const void *x_fp16,
         ranges_overlap(workspace, need, x_fp16, static_cast<size_t>(M) * h->K * 2))
         return fail(PTQ_ERR_VALUE, "workspace overlaps x or y");
     if ((st = launch_quantize(h, x_fp16, M, workspace, h->Kpad, s)) != PTQ_OK) return st;
-    if ((st = launch_gemm_any(h, workspace, M, y_fp16, acc_int32_out, s)) != PTQ_OK) return st;
+    if ((st = launch_gemm_any(h, workspace, M, y_fp16, acc_int32_out, s, (flags & PTQ_FLAG_CTA_PAIR) != 0)) != PTQ_OK)
+        return st;
     if (q_int8_out)
         PTQ_CUDA(cudaMemcpy2DAsync(q_int8_out, h->K, workspace, h->Kpad, h->K, static_cast<size_t>(M),
                                    cudaMemcpyDeviceToDevice, s));

@@ -41,9 +41,9 @@ def layer_inputs(spec, B=None):
     return x, wq, dw, bias, s, dx
 
 
-def check_layer(ptq, torch, spec, B=None, flags_list=(0, 1), full=None, seed=0):
+def check_layer(ptq, torch, spec, B=None, flags_list=(0, 1, 2), full=None, seed=0):
     """Forward with taps through the C ABI, once per entry of flags_list (0 = quantize kernel then
-    GEMM kernel, 1 = PTQ_FLAG_FUSED_PROLOGUE); compare codes and accumulators bit for bit and the fp16
+    GEMM kernel, 1 = PTQ_FLAG_FUSED_PROLOGUE, 2 = PTQ_FLAG_CTA_PAIR); compare codes and accumulators bit for bit and the fp16
     output within tolerance, on every row (small layers) or on sampled row blocks (large ones)."""
     x, wq, dw, bias, s, dx = layer_inputs(spec, B)
     Bn = x.shape[0]
