@@ -152,50 +152,57 @@ __device__ __forceinline__ void store_acc32(const uint32_t (&v)[32], int32_t *ar
 }
 
 // Epilogue of one 128 x BN accumulator for one warp (its 32-lane quarter).  `tmem_row` addresses the
-// warp's lanes and the accumulator's first column.  Returns the updated count of staged boxes.
-template <bool kDebugAcc>
+// warp's lanes and the accumulator's first column.  The warp takes every second 64-column box
+// (`col_half` selects which).  Returns the updated count of staged boxes.
+// kLowReg = false loads the box's 64 columns with two TMEM loads in flight (64 accumulator registers);
+// kLowReg = true converts 32 columns at a time (for kernels whose thread count caps the registers).
+template <bool kDebugAcc, bool kLowReg = false>
 __device__ __forceinline__ uint32_t epilogue_tile(const GemmParams &p, const CUtensorMap *tmY, uint32_t tmem_row,
                                                   long long m_row0, int n0, float dxr, uint32_t staging,
                                                   uint32_t nboxes, int lane, int col_half)
 {
     const long long m = m_row0 + lane;
     const bool row_ok = m < p.M;
+    const uint32_t row_addr = staging + static_cast<uint32_t>(lane) * 128u;
     for (int c0 = col_half * kStoreBoxCols; c0 < p.BN; c0 += 2 * kStoreBoxCols) {
+        const int n_first = n0 + c0;
         uint32_t v0[32], v1[32];
         tmem_ld_32x32(tmem_row + c0, v0);
-        tmem_ld_32x32(tmem_row + c0 + 32, v1);
+        if (!kLowReg) tmem_ld_32x32(tmem_row + c0 + 32, v1);
         tmem_ld_wait();
-        const int n_first = n0 + c0;
-        if (kDebugAcc) {
-            if (p.acc_out != nullptr && row_ok) {
-                store_acc32(v0, p.acc_out + m * p.N, n_first, p.N);
-                store_acc32(v1, p.acc_out + m * p.N, n_first + 32, p.N);
+        if (p.use_tma_store) {
+            if (nboxes >= 1u && lane == 0) bulk_wait_group_read<0>();   // the previous box has left the buffer
+            __syncwarp();
+        }
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            uint32_t (&v)[32] = (half == 0 || kLowReg) ? v0 : v1;
+            if (kLowReg && half == 1) {
+                tmem_ld_32x32(tmem_row + c0 + 32, v0);
+                tmem_ld_wait();
+            }
+            const int n_half = n_first + 32 * half;
+            if (kDebugAcc) {
+                if (p.acc_out != nullptr && row_ok) store_acc32(v, p.acc_out + m * p.N, n_half, p.N);
+            }
+            if (p.use_tma_store) {
+                convert_stage32(v, half, dxr, p.dw + n_half, p.bias + n_half, row_addr, lane);
+            } else if (row_ok && p.y_vec8) {
+                convert_store32_vec8(v, dxr, p.dw + n_half, p.bias + n_half, p.y + m * p.N, n_half, p.N);
+            } else if (row_ok) {
+                convert_store32_plain(v, dxr, p.dw + n_half, p.bias + n_half, p.y + m * p.N, n_half, p.N,
+                                      p.y_vec2 != 0);
             }
         }
         if (p.use_tma_store) {
-            const uint32_t buf = staging;
-            if (nboxes >= 1u && lane == 0) bulk_wait_group_read<0>();   // the previous box has left the buffer
-            __syncwarp();
-            const uint32_t row_addr = buf + static_cast<uint32_t>(lane) * 128u;
-            convert_stage32(v0, 0, dxr, p.dw + n_first, p.bias + n_first, row_addr, lane);
-            convert_stage32(v1, 1, dxr, p.dw + n_first + 32, p.bias + n_first + 32, row_addr, lane);
             fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) {
                 if (n_first < p.N && m_row0 < p.M)
-                    tma_store_2d(tmY, n_first, static_cast<int>(m_row0), buf);   // clipped at N and M
+                    tma_store_2d(tmY, n_first, static_cast<int>(m_row0), staging);   // clipped at N and M
                 bulk_commit_group();
             }
             ++nboxes;
-        } else if (row_ok && p.y_vec8) {
-            __half *yrow = p.y + m * p.N;
-            convert_store32_vec8(v0, dxr, p.dw + n_first, p.bias + n_first, yrow, n_first, p.N);
-            convert_store32_vec8(v1, dxr, p.dw + n_first + 32, p.bias + n_first + 32, yrow, n_first + 32, p.N);
-        } else if (row_ok) {
-            __half *yrow = p.y + m * p.N;
-            convert_store32_plain(v0, dxr, p.dw + n_first, p.bias + n_first, yrow, n_first, p.N, p.y_vec2 != 0);
-            convert_store32_plain(v1, dxr, p.dw + n_first + 32, p.bias + n_first + 32, yrow, n_first + 32, p.N,
-                                  p.y_vec2 != 0);
         }
     }
     return nboxes;
