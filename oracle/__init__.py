@@ -40,11 +40,8 @@ def build(force: bool = False) -> str:
     return _SO
 
 
-def lib() -> ctypes.CDLL:
-    global _lib
-    if _lib is not None:
-        return _lib
-    L = ctypes.CDLL(build())
+def _bind(path: str) -> ctypes.CDLL:
+    L = ctypes.CDLL(path)
     c_long, c_int, vp = ctypes.c_long, ctypes.c_int, ctypes.c_void_p
     L.ptqo_num_threads.restype = c_int
     L.ptqo_half_to_float.restype = ctypes.c_float
@@ -64,8 +61,38 @@ def lib() -> ctypes.CDLL:
                                            vp, vp, vp, vp, vp, vp, vp, vp]
     L.ptqo_calibrate.restype = None
     L.ptqo_calibrate.argtypes = [vp, c_int, c_int, c_int, vp, vp, c_int, vp, vp]
-    _lib = L
     return L
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        _lib = _bind(build())
+    return _lib
+
+
+class use_library:
+    """Context manager for the tests of the tests: run the oracle's Python API against another build of
+    ``ptq_oracle.c`` (a copy with a planted mistake) to show that the pins notice it."""
+
+    def __init__(self, source_text: str, workdir: str):
+        self.src = os.path.join(workdir, "ptq_oracle_mutant.c")
+        self.so = os.path.join(workdir, "libptq_oracle_mutant_%d.so" % (abs(hash(source_text)) % 10 ** 9))
+        with open(self.src, "w") as f:
+            f.write(source_text)
+        subprocess.run(["gcc", "-O2", "-fopenmp", "-ffp-contract=off", "-fno-fast-math", "-std=c99",
+                        "-D_DEFAULT_SOURCE", "-shared", "-fPIC", self.src, "-o", self.so, "-lm"], check=True)
+
+    def __enter__(self):
+        global _lib
+        self.saved = lib()
+        _lib = _bind(self.so)
+        return self
+
+    def __exit__(self, *exc):
+        global _lib
+        _lib = self.saved
+        return False
 
 
 def _p(a):

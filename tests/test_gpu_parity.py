@@ -79,6 +79,66 @@ def test_quantizer_all_fp16_inputs_many_scales(env):
         assert np.array_equal(q, want)
 
 
+def test_quantizer_tie_adjacent_inputs_all_paths(env):
+    # x = fp16((j + 0.5) s[k] dx[t]) for every half-integer j + 0.5 in [-127.5, 127.5]: the quotient lands
+    # within fp16 rounding of a tie, so a large share of the elements falls inside the screening band and
+    # is decided by the exact two-division route.  Checked for the quantize kernel and, through the
+    # accumulators, for the fused kernel's in-kernel quantizers.
+    ptq, torch = env
+    rng = np.random.default_rng(14)
+    T, K, N = 16, 64, 16
+    s = np.exp(rng.uniform(np.log(5e-2), np.log(2e1), K)).astype(np.float32)
+    dx = np.exp(rng.uniform(np.log(1e-2), np.log(1.0), T)).astype(np.float32)
+    j = (np.arange(256) - 128 + 0.5)
+    x = (j[:, None, None] * (s.astype(np.float64)[None, None, :] * dx.astype(np.float64)[None, :, None])).astype(np.float16)
+    x = np.concatenate([x, np.nextafter(x, np.float16(np.inf)), np.nextafter(x, np.float16(-np.inf))], axis=0)
+    B = x.shape[0]
+    wq = rng.integers(-127, 128, (N, K)).astype(np.int8)
+    layer = ptq.PtqLinear(wq, np.full(N, 0.01, np.float32), s, dx)
+    xd = torch.from_numpy(x).cuda()
+    q_ref = oracle.quantize(x.reshape(-1, K), T, s, dx)
+    q = layer.quantize(xd).cpu().numpy().reshape(-1, K)
+    assert np.array_equal(q, q_ref)
+    acc_ref = oracle.int_matmul(q_ref, wq)
+    for flags in (0, ptq.FLAG_FUSED_PROLOGUE):
+        _, q2, acc = layer.forward_debug(xd, flags=flags)
+        torch.cuda.synchronize()
+        layer.device_status()
+        assert np.array_equal(q2.cpu().numpy().reshape(-1, K), q_ref)
+        assert np.array_equal(acc.cpu().numpy().reshape(B * T, N), acc_ref)
+    # how many elements actually sat inside the band (exact quotient within 6e-5 of a tie)
+    v = x.astype(np.float64) / s.astype(np.float64)[None, None, :] / dx.astype(np.float64)[None, :, None]
+    inside = np.abs(np.abs(v - np.floor(v)) - 0.5) < 6e-5
+    assert inside.mean() > 0.02
+
+
+def test_forward_edge_arguments(env):
+    ptq, torch = env
+    spec = CFG[0][0]
+    x, wq, dw, bias, s, dx = layer_inputs(spec, B=1)
+    layer = ptq.PtqLinear(wq, dw, s, dx, bias)
+    L = ptq.load_library()
+    xd = torch.from_numpy(x).cuda()
+    y = torch.empty((1, spec.T, spec.N), dtype=torch.float16, device="cuda")
+    ws = torch.empty(layer.workspace_bytes(1), dtype=torch.uint8, device="cuda")
+    for B in (0, -3):                                  # an empty batch is refused, nothing is launched
+        n0 = ptq.binding.kernel_launch_count()
+        assert L.ptq_linear_forward(layer._h, xd.data_ptr(), B, y.data_ptr(), ws.data_ptr(), ws.numel(), 0, None) == 2
+        assert L.ptq_quantize(layer._h, xd.data_ptr(), B, ws.data_ptr(), None) == 2
+        assert ptq.binding.kernel_launch_count() == n0
+    assert layer.workspace_bytes(0) == 0
+    assert L.ptq_linear_forward(layer._h, xd.data_ptr(), 1, xd.data_ptr(), ws.data_ptr(), ws.numel(), 0, None) == 3   # y aliases x
+    assert L.ptq_linear_forward(layer._h, xd.data_ptr(), 1, y.data_ptr(), ws.data_ptr() + 8, ws.numel() - 8, 0, None) in (2, 4)
+    assert "K=384 N=192" in layer.describe()
+
+
+@pytest.mark.parametrize("K,N,T,B", [(16, 65536, 3, 3), (8, 24, 100003, 1), (8192, 8, 1, 300)])
+def test_maximum_sizes(env, K, N, T, B):
+    ptq, torch = env
+    spec = wl.LinearSpec(8, 1, 1, "max", B, T, K, N, bias=True, n_outliers=1)
+    check_layer(ptq, torch, spec, full=True)
+
+
 def test_quantizer_scales_outside_reciprocal_range_use_ieee_division(env):
     ptq, torch = env
     rng = np.random.default_rng(12)

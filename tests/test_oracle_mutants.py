@@ -1,0 +1,89 @@
+"""Tests of the pins themselves.  Each case plants one plausible mistake in a COPY of the oracle's C
+source (a dropped term, a wrong sign or index, a transposed operand, a wrong rounding), builds it, and
+requires that at least one pin of test_oracle_pins.py fails against it.  Everything runs on the CPU."""
+import os
+
+import pytest
+
+import oracle
+import test_oracle_pins as pins
+
+SRC = open(os.path.join(os.path.dirname(oracle.__file__), "ptq_oracle.c")).read()
+
+# (name, text to find, replacement, pins expected to notice)
+MUTANTS = [
+    ("truncate instead of round-to-nearest", "r = nearbyintf(v);", "r = truncf(v);",
+     [lambda: pins.test_quantizer_ties_clamp_and_specials()]),
+    ("ties away from zero", "r = nearbyintf(v);", "r = roundf(v);",
+     [lambda: pins.test_quantizer_ties_clamp_and_specials()]),
+    ("clamp to the symmetric range", "if (r < -128.0f) r = -128.0f;", "if (r < -127.0f) r = -127.0f;",
+     [lambda: pins.test_quantizer_ties_clamp_and_specials()]),
+    ("NaN not mapped to zero", "if (isnan(v)) return 0;", "if (isnan(v)) return 127;",
+     [lambda: pins.test_quantizer_ties_clamp_and_specials()]),
+    ("multiply by s instead of dividing", "volatile float u = xf / s;", "volatile float u = xf * s;",
+     [lambda: pins.test_quantizer_indexes_token_position_and_channel()]),
+    ("one fused division", "volatile float v = u / dx;", "volatile float v = xf / (s * dx);",
+     [lambda: pins.test_quantizer_keeps_the_two_divisions_separate()]),
+    ("reciprocal multiplications instead of divisions", "volatile float u = xf / s;\n    volatile float v = u / dx;",
+     "volatile float rs_ = 1.0f / s; volatile float rd_ = 1.0f / dx; volatile float u = xf * rs_;\n    volatile float v = u * rd_;",
+     [lambda: pins.test_quantizer_keeps_the_two_divisions_separate()]),
+    ("step indexed by row instead of token position", "q[m * K + k] = ptqo_quantize_one(x[m * K + k], s[k], dx[t]);",
+     "q[m * K + k] = ptqo_quantize_one(x[m * K + k], s[k], dx[m % 2]);",
+     [lambda: pins.test_quantizer_indexes_token_position_and_channel()]),
+    ("smoothing scale of the wrong channel", "q[m * K + k] = ptqo_quantize_one(x[m * K + k], s[k], dx[t]);",
+     "q[m * K + k] = ptqo_quantize_one(x[m * K + k], s[(k + 1) % K], dx[t]);",
+     [lambda: pins.test_quantizer_indexes_token_position_and_channel()]),
+    ("transposed weight in the contraction", "sum += (int64_t)q[m * K + k] * (int64_t)wq[(long)n * K + k];\n            if (sum > INT32_MAX || sum < INT32_MIN) overflow = 1;\n            acc[m * N + n]",
+     "sum += (int64_t)q[m * K + k] * (int64_t)wq[((long)k * N + n) % ((long)N * K)];\n            if (sum > INT32_MAX || sum < INT32_MIN) overflow = 1;\n            acc[m * N + n]",
+     [lambda: pins.test_int_matmul_brute_force_tiny()]),
+    ("last term of the contraction dropped", "for (k = 0; k < K; ++k)\n                sum += (int64_t)q[m * K + k] * (int64_t)wq[(long)n * K + k];\n            if (sum > INT32_MAX || sum < INT32_MIN) overflow = 1;\n            acc[m * N + n]",
+     "for (k = 0; k + 1 < K; ++k)\n                sum += (int64_t)q[m * K + k] * (int64_t)wq[(long)n * K + k];\n            if (sum > INT32_MAX || sum < INT32_MIN) overflow = 1;\n            acc[m * N + n]",
+     [lambda: pins.test_int_matmul_one_hot_and_extremes()]),
+    ("dequant forgets the activation step", "double yd = (double)acc[m * N + n] * (double)dx[t] * (double)dw[n];",
+     "double yd = (double)acc[m * N + n] * (double)dw[n];",
+     [lambda: pins.test_dequant_power_of_two_steps_exact()]),
+    ("dequant uses the weight step of the row", "double yd = (double)acc[m * N + n] * (double)dx[t] * (double)dw[n];",
+     "double yd = (double)acc[m * N + n] * (double)dx[t] * (double)dw[m % N];",
+     [lambda: pins.test_dequant_power_of_two_steps_exact()]),
+    ("bias subtracted", "if (bias) yd += (double)bias[n];\n            y[m * N + n]", "if (bias) yd -= (double)bias[n];\n            y[m * N + n]",
+     [lambda: pins.test_dequant_equals_product_of_dequantized_operands()]),
+    ("half conversion rounds toward zero", "double m = nearbyint(ldexp(f, 11));", "double m = floor(ldexp(f, 11));",
+     [lambda: pins.test_double_to_half_roundtrip_and_midpoints()]),
+    ("overflow saturates to the largest half", "if (a >= 65520.0) return (uint16_t)(sign | 0x7c00);",
+     "if (a >= 65520.0) return (uint16_t)(sign | 0x7bff);",
+     [lambda: pins.test_double_to_half_roundtrip_and_midpoints()]),
+    ("subnormal halves decoded with the wrong scale", "v = ldexpf((float)frac, -24);", "v = ldexpf((float)frac, -25);",
+     [lambda: pins.test_half_to_float_all_patterns()]),
+    ("fused forward drops the bias", "if (bias) yd += (double)bias[n];\n            y[(m - m0) * N + n]",
+     "y[(m - m0) * N + n]", [lambda: pins.test_forward_rows_equals_composition_and_row_ranges()]),
+    ("fused forward ignores the row offset", "y[(m - m0) * N + n] = ptqo_double_to_half(yd);",
+     "y[((m - m0) * N + n + 1) % ((m1 - m0) * N)] = ptqo_double_to_half(yd);",
+     [lambda: pins.test_forward_rows_equals_composition_and_row_ranges()]),
+    ("smoothing scale without the square root", "s[k] = sqrtf(ratio);", "s[k] = ratio;",
+     [lambda: pins.test_calibrate_vs_numpy_float32_and_no_clip_invariant()]),
+    ("calibration divides by 128", "volatile float d = mu / 127.0f;", "volatile float d = mu / 128.0f;",
+     [lambda: pins.test_calibrate_vs_numpy_float32_and_no_clip_invariant()]),
+    ("weight magnitude ignores the weight step", "volatile float a = fabsf((float)wq[(long)n * K + k]) * dw[n];",
+     "volatile float a = fabsf((float)wq[(long)n * K + k]);",
+     [lambda: pins.test_calibrate_degenerate_channels_and_positions()]),
+    ("calibration without the floor", "if (mu < floor_) mu = floor_;", "",
+     [lambda: pins.test_calibrate_degenerate_channels_and_positions()]),
+]
+
+
+@pytest.mark.parametrize("name,find,repl,checks", MUTANTS, ids=[m[0] for m in MUTANTS])
+def test_planted_mistake_is_caught_by_a_pin(tmp_path, name, find, repl, checks):
+    assert SRC.count(find) == 1, "mutation site not found exactly once: %s" % name
+    with oracle.use_library(SRC.replace(find, repl), str(tmp_path)):
+        caught = 0
+        for check in checks:
+            try:
+                check()
+            except AssertionError:
+                caught += 1
+            except OverflowError:
+                caught += 1
+        assert caught >= 1, "no pin noticed: %s" % name
+    # and the unmodified oracle passes the same checks
+    for check in checks:
+        check()

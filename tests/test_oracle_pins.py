@@ -119,6 +119,35 @@ def test_quantizer_vs_float64_differs_only_near_ties():
     assert total_diff < 200
 
 
+def test_quantizer_keeps_the_two_divisions_separate():
+    # (x/s)/dx, x/(s*dx) and x*(1/s)*(1/dx) agree except within an ulp of a rounding tie.  Search for
+    # inputs where the binary32 results of these formulations give different codes and require the
+    # oracle to side with the two-division definition on every one of them.
+    rng = np.random.default_rng(21)
+    n = 20000
+    xh = (rng.standard_normal(n) * 10.0 ** rng.uniform(-2, 2, n)).astype(np.float16)
+    xh = xh[np.isfinite(xh) & (xh != 0)]
+    xf = xh.astype(F32)
+    s = np.exp(rng.uniform(np.log(1e-2), np.log(1e2), xf.size)).astype(F32)
+    k = rng.integers(1, 127, xf.size).astype(F32) + F32(0.5)
+    u = (xf / s).astype(F32)
+    found = []
+    for nudge in (-2, -1, 0, 1, 2):                       # steps chosen so that the quotient lands next to a tie
+        dx = (np.abs(u) / k).astype(F32)
+        for _ in range(abs(nudge)):
+            dx = np.nextafter(dx, F32(np.inf) if nudge > 0 else F32(0)).astype(F32)
+        ok = np.isfinite(dx) & (dx > 0)
+        two = np.clip(np.rint((xf / s).astype(F32) / dx), -128, 127)
+        one = np.clip(np.rint(xf / (s * dx).astype(F32)), -128, 127)
+        rec = np.clip(np.rint((xf * (F32(1) / s).astype(F32)).astype(F32) * (F32(1) / dx).astype(F32)), -128, 127)
+        for idx in np.nonzero(ok & ((two != one) | (two != rec)))[0][:60]:
+            found.append((xh[idx], s[idx], dx[idx], int(two[idx])))
+    assert len(found) >= 40, "search found too few discriminating inputs (%d)" % len(found)
+    for x, s, dx, want in found:
+        got = oracle.quantize_one(int(np.float16(x).view(np.uint16)), float(s), float(dx))
+        assert got == want, (float(x), float(s), float(dx), got, want)
+
+
 def test_quantizer_ties_clamp_and_specials():
     one = np.array([1.0], F32)
 
