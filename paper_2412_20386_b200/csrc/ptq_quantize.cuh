@@ -75,15 +75,16 @@ __device__ __forceinline__ float dist_to_integer(float v)
 // distance-to-tie test.  Returns true when one of the 8 values sits within the error bound of a
 // rounding tie, in which case the caller recomputes the 8 codes with the two exact divisions.
 // Values beyond +-127.5 clamp to the same code whichever way a tie falls, NaN converts to 0 and
-// infinities saturate on both routes, so a needless trip through the exact route (NaN, inf and huge
-// values fail the test) costs time only: the final codes are always those of the definition.
+// infinities saturate on both routes, so whether such values pass the test or not only costs time:
+// the final codes are always those of the definition.
 // Valid only when every scale lies in [2^-30, 2^30] (no under/overflow in c or x * c).
 __device__ __forceinline__ bool quantize8_screen(uint32_t x0, uint32_t x1, uint32_t x2, uint32_t x3,
                                                  const float (&c8)[8], uint32_t &lo, uint32_t &hi)
 {
     const uint32_t xw[4] = {x0, x1, x2, x3};
     int c[8];
-    bool near_tie = false;
+    float worst = 0.0f;   // largest distance to an integer; fmaxf drops the NaN that NaN / inf inputs produce,
+                          // which is fine: their codes (0, +-saturation) are the same on both routes
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         __half2 h = *reinterpret_cast<const __half2 *>(&xw[i]);
@@ -92,12 +93,11 @@ __device__ __forceinline__ bool quantize8_screen(uint32_t x0, uint32_t x1, uint3
         const float v1 = __fmul_rn(f.y, c8[2 * i + 1]);
         c[2 * i] = f32_to_code(v0);
         c[2 * i + 1] = f32_to_code(v1);
-        near_tie = near_tie || !(dist_to_integer(v0) <= kScreenThreshold);
-        near_tie = near_tie || !(dist_to_integer(v1) <= kScreenThreshold);
+        worst = fmaxf(worst, fmaxf(dist_to_integer(v0), dist_to_integer(v1)));
     }
     lo = pack4(c[0], c[1], c[2], c[3]);
     hi = pack4(c[4], c[5], c[6], c[7]);
-    return near_tie;
+    return worst > kScreenThreshold;
 }
 
 // Exact route for the same 8 channels: two correctly rounded divisions per element.  s8 / rs8 point
