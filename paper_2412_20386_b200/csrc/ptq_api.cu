@@ -64,22 +64,24 @@ encode_tiled_fn get_encode_tiled()
 }
 
 // 2-D row-major tensor [rows, cols] with `pitch_bytes` between rows; box [box_rows, box_cols];
-// 128-byte swizzle (box_cols * elem_bytes must be 128); out-of-range elements read as zero and
-// are skipped on stores.
+// the swizzle mode follows the box's row bytes (128 or 64, which box_cols * elem_bytes must equal);
+// out-of-range elements read as zero and are skipped on stores.
 ptq_status_t make_map_2d(CUtensorMap *map, CUtensorMapDataType dt, int elem_bytes, const void *ptr,
                          unsigned long long cols, unsigned long long rows, unsigned long long pitch_bytes,
                          unsigned box_cols, unsigned box_rows)
 {
     encode_tiled_fn enc = get_encode_tiled();
     if (!enc) return fail(PTQ_ERR_CUDA, "cuTensorMapEncodeTiled entry point not available");
-    if (box_cols * elem_bytes != 128 || box_rows == 0 || box_rows > 256)
+    const unsigned row_bytes = box_cols * elem_bytes;
+    if ((row_bytes != 128 && row_bytes != 64) || box_rows == 0 || box_rows > 256)
         return fail(PTQ_ERR_SHAPE, "internal: bad TMA box %u x %u", box_rows, box_cols);
     cuuint64_t dims[2] = {cols, rows};
     cuuint64_t strides[1] = {pitch_bytes};
     cuuint32_t box[2] = {box_cols, box_rows};
     cuuint32_t estr[2] = {1, 1};
     CUresult r = enc(map, dt, 2, const_cast<void *>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     row_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS)
         return fail(PTQ_ERR_CUDA, "cuTensorMapEncodeTiled failed with CUresult %d (cols %llu rows %llu pitch %llu)",

@@ -13,8 +13,8 @@
 //   warp 1      owns TMEM (512 columns = two 128 x 256 accumulators) and issues the MMAs; a
 //               tcgen05.commit frees each shared-memory stage and publishes each accumulator
 //   warps 2..9  epilogue: tcgen05.ld (lane quarter = warp % 4; the two warps of a quarter take
-//               alternate 64-column boxes), scale, convert, stage the fp16 box in swizzled shared
-//               memory and write it with a TMA store
+//               alternate 64-column steps), scale, convert, stage 32 x 32 fp16 boxes in swizzled shared
+//               memory (two per warp) and write them with TMA stores
 // While the epilogue drains accumulator i the MMA warp already fills accumulator i^1.
 #pragma once
 
@@ -33,9 +33,10 @@ constexpr int kATileBytes = kBM * kBK;                    // 16 KB
 constexpr int kBTileBytes = kMaxBN * kBK;                 // 32 KB
 constexpr int kStageBytes = kATileBytes + kBTileBytes;
 constexpr int kNumEpiWarps = 8;                           // two per TMEM lane quarter
-constexpr int kStoreBoxCols = 64;                         // fp16 columns per TMA store box (128 B)
-constexpr int kStoreBoxBytes = 32 * kStoreBoxCols * 2;    // 32 rows x 128 B
-constexpr int kStagingBytesPerWarp = kStoreBoxBytes;      // reused once the previous box has been read
+constexpr int kEpiStepCols = 64;                          // accumulator columns a warp drains per step
+constexpr int kStoreBoxCols = 32;                         // fp16 columns per TMA store box (64-byte rows)
+constexpr int kStoreBoxBytes = 32 * kStoreBoxCols * 2;    // 32 rows x 64 B = 2 KB
+constexpr int kStagingBytesPerWarp = 2 * kStoreBoxBytes;  // two boxes: one being filled while the other is stored
 constexpr int kGemmThreads = 32 * (2 + kNumEpiWarps);
 constexpr int kTmemCols = 512;
 constexpr int kNumBarriers = 2 * kStages + 4;
@@ -80,12 +81,13 @@ __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint4 v)
                  : "memory");
 }
 
-// Convert 32 accumulator columns of this thread's row and write them as four 16-byte chunks of the
-// row's 128-byte line in the staging buffer (chunk index XOR (row & 7): the 128-byte swizzle the
-// store's tensor map expects, which also spreads the 32 rows over all banks).
-__device__ __forceinline__ void convert_stage32(const uint32_t (&v)[32], int half, float dxr, const float *dw,
+// Convert 32 accumulator columns of this thread's row and write them as the four 16-byte chunks of the
+// row's 64-byte line in a staging box (chunk index XOR ((row >> 1) & 3): the 64-byte swizzle the store's
+// tensor map expects, which also spreads the 32 rows over all banks).
+__device__ __forceinline__ void convert_stage32(const uint32_t (&v)[32], float dxr, const float *dw,
                                                 const float *bias, uint32_t row_addr, int lane)
 {
+    const uint32_t sw = static_cast<uint32_t>((lane >> 1) & 3);
 #pragma unroll
     for (int jj = 0; jj < 4; ++jj) {
         const float4 w0 = __ldg(reinterpret_cast<const float4 *>(dw + 8 * jj));
@@ -97,8 +99,7 @@ __device__ __forceinline__ void convert_stage32(const uint32_t (&v)[32], int hal
         o.y = pack_half2(dequant_one(v[8 * jj + 2], dxr, w0.z, b0.z), dequant_one(v[8 * jj + 3], dxr, w0.w, b0.w));
         o.z = pack_half2(dequant_one(v[8 * jj + 4], dxr, w1.x, b1.x), dequant_one(v[8 * jj + 5], dxr, w1.y, b1.y));
         o.w = pack_half2(dequant_one(v[8 * jj + 6], dxr, w1.z, b1.z), dequant_one(v[8 * jj + 7], dxr, w1.w, b1.w));
-        const int chunk = half * 4 + jj;
-        st_shared_v4(row_addr + (static_cast<uint32_t>(chunk ^ (lane & 7)) << 4), o);
+        st_shared_v4(row_addr + ((static_cast<uint32_t>(jj) ^ sw) << 4), o);
     }
 }
 
@@ -152,10 +153,12 @@ __device__ __forceinline__ void store_acc32(const uint32_t (&v)[32], int32_t *ar
 }
 
 // Epilogue of one 128 x BN accumulator for one warp (its 32-lane quarter).  `tmem_row` addresses the
-// warp's lanes and the accumulator's first column.  The warp takes every second 64-column box
-// (`col_half` selects which).  Returns the updated count of staged boxes.
-// kLowReg = false loads the box's 64 columns with two TMEM loads in flight (64 accumulator registers);
-// kLowReg = true converts 32 columns at a time (for kernels whose thread count caps the registers).
+// warp's lanes and the accumulator's first column.  The warp takes every second 64-column step
+// (`col_half` selects which) and writes each step as two 32-column boxes; with two staging boxes per
+// warp a TMA store is still reading one box while the next is being filled, so the latency of a store
+// is not on the warp's critical path.  Returns the updated count of staged boxes.
+// kLowReg = false keeps both TMEM loads of a step in flight (64 accumulator registers);
+// kLowReg = true loads 32 columns at a time (for kernels whose thread count caps the registers).
 template <bool kDebugAcc, bool kLowReg = false>
 __device__ __forceinline__ uint32_t epilogue_tile(const GemmParams &p, const CUtensorMap *tmY, uint32_t tmem_row,
                                                   long long m_row0, int n0, float dxr, uint32_t staging,
@@ -163,17 +166,12 @@ __device__ __forceinline__ uint32_t epilogue_tile(const GemmParams &p, const CUt
 {
     const long long m = m_row0 + lane;
     const bool row_ok = m < p.M;
-    const uint32_t row_addr = staging + static_cast<uint32_t>(lane) * 128u;
-    for (int c0 = col_half * kStoreBoxCols; c0 < p.BN; c0 += 2 * kStoreBoxCols) {
+    for (int c0 = col_half * kEpiStepCols; c0 < p.BN; c0 += 2 * kEpiStepCols) {
         const int n_first = n0 + c0;
         uint32_t v0[32], v1[32];
         tmem_ld_32x32(tmem_row + c0, v0);
         if (!kLowReg) tmem_ld_32x32(tmem_row + c0 + 32, v1);
         tmem_ld_wait();
-        if (p.use_tma_store) {
-            if (nboxes >= 1u && lane == 0) bulk_wait_group_read<0>();   // the previous box has left the buffer
-            __syncwarp();
-        }
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
             uint32_t (&v)[32] = (half == 0 || kLowReg) ? v0 : v1;
@@ -186,23 +184,24 @@ __device__ __forceinline__ uint32_t epilogue_tile(const GemmParams &p, const CUt
                 if (p.acc_out != nullptr && row_ok) store_acc32(v, p.acc_out + m * p.N, n_half, p.N);
             }
             if (p.use_tma_store) {
-                convert_stage32(v, half, dxr, p.dw + n_half, p.bias + n_half, row_addr, lane);
+                const uint32_t box = staging + (nboxes & 1u) * kStoreBoxBytes;
+                if (nboxes >= 2u && lane == 0) bulk_wait_group_read<1>();   // the store that last used this box has read it
+                __syncwarp();
+                convert_stage32(v, dxr, p.dw + n_half, p.bias + n_half, box + static_cast<uint32_t>(lane) * 64u, lane);
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    if (n_half < p.N && m_row0 < p.M)
+                        tma_store_2d(tmY, n_half, static_cast<int>(m_row0), box);   // clipped at N and M
+                    bulk_commit_group();
+                }
+                ++nboxes;
             } else if (row_ok && p.y_vec8) {
                 convert_store32_vec8(v, dxr, p.dw + n_half, p.bias + n_half, p.y + m * p.N, n_half, p.N);
             } else if (row_ok) {
                 convert_store32_plain(v, dxr, p.dw + n_half, p.bias + n_half, p.y + m * p.N, n_half, p.N,
                                       p.y_vec2 != 0);
             }
-        }
-        if (p.use_tma_store) {
-            fence_proxy_async_smem();
-            __syncwarp();
-            if (lane == 0) {
-                if (n_first < p.N && m_row0 < p.M)
-                    tma_store_2d(tmY, n_first, static_cast<int>(m_row0), staging);   // clipped at N and M
-                bulk_commit_group();
-            }
-            ++nboxes;
         }
     }
     return nboxes;
