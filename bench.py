@@ -438,10 +438,10 @@ def run_ours(args, specs, rank, world, local_rank):
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised
 # under profiles/; keyed by (kernel, workload, layer).  An entry is removed when its kernel changes.
 TRAFFIC = {
-    ("ptq_gemm_dequant_kernel", "c3", "in_proj"): 41.172992e6 + 250.858496e6,
-    ("ptq_gemm_dequant_kernel", "c3", "out_proj"): 78.695424e6 + 32.746496e6,
-    ("ptq_quantize_kernel", "c3", "in_proj"): 77.500160e6 + 6.917376e6,
-    ("ptq_quantize_kernel", "c3", "out_proj"): 154.963968e6 + 24.366080e6,
+    ("ptq_gemm_dequant_kernel", "c3", "in_proj"): 41.241088e6 + 255.717632e6,
+    ("ptq_gemm_dequant_kernel", "c3", "out_proj"): 78.695936e6 + 34.413312e6,
+    ("ptq_quantize_kernel", "c3", "in_proj"): 77.491456e6 + 7.729664e6,
+    ("ptq_quantize_kernel", "c3", "out_proj"): 154.964736e6 + 24.675072e6,
 }
 
 
