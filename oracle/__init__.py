@@ -61,6 +61,17 @@ def _bind(path: str) -> ctypes.CDLL:
                                            vp, vp, vp, vp, vp, vp, vp, vp]
     L.ptqo_calibrate.restype = None
     L.ptqo_calibrate.argtypes = [vp, c_int, c_int, c_int, vp, vp, c_int, vp, vp]
+    L.ptqo_quantize_asym_one.restype = ctypes.c_uint8
+    L.ptqo_quantize_asym_one.argtypes = [ctypes.c_uint16, ctypes.c_float, ctypes.c_float, c_int]
+    L.ptqo_quantize_asym.restype = None
+    L.ptqo_quantize_asym.argtypes = [vp, c_long, c_int, c_int, vp, vp, vp, vp]
+    L.ptqo_int_matmul_asym.restype = c_int
+    L.ptqo_int_matmul_asym.argtypes = [vp, vp, c_int, vp, c_long, c_int, c_int, vp]
+    L.ptqo_calibrate_asym.restype = None
+    L.ptqo_calibrate_asym.argtypes = [vp, c_int, c_int, c_int, vp, vp, c_int, vp, vp, vp]
+    L.ptqo_linear_forward_rows_asym.restype = c_int
+    L.ptqo_linear_forward_rows_asym.argtypes = [vp, c_long, c_long, c_int, c_int, c_int,
+                                                vp, vp, vp, vp, vp, vp, vp, vp, vp]
     return L
 
 
@@ -206,3 +217,80 @@ def calibrate(xcal, wq, dw):
     dx = np.empty(T, np.float32)
     lib().ptqo_calibrate(_p(xcal), Bc, T, K, _p(wq), _p(dw), N, _p(s), _p(dx))
     return s, dx
+
+
+# --------------------------------------------------------------------------- #
+# asymmetric PTS (step and zero offset per token position)                     #
+# --------------------------------------------------------------------------- #
+def quantize_asym_one(x_bits: int, s: float, dx: float, z: int) -> int:
+    return int(lib().ptqo_quantize_asym_one(int(x_bits), float(s), float(dx), int(z)))
+
+
+def quantize_asym(x, T, s, dx, z):
+    """x fp16 [M,K] -> uint8 codes [M,K] = clip(round((x/s)/dx[t]) + z[t], 0, 255)."""
+    x = _c(x, np.float16)
+    M, K = x.shape
+    s = _c(s, np.float32)
+    dx = _c(dx, np.float32)
+    z = _c(z, np.int32)
+    assert s.shape == (K,) and dx.shape == (T,) and z.shape == (T,)
+    c = np.empty((M, K), np.uint8)
+    lib().ptqo_quantize_asym(_p(x), M, K, T, _p(s), _p(dx), _p(z), _p(c))
+    return c
+
+
+def int_matmul_asym(c, z, T, wq):
+    """acc[m,n] = sum_k (c[m,k] - z[m mod T]) * wq[n,k] (raises on int32 overflow)."""
+    c = _c(c, np.uint8)
+    z = _c(z, np.int32)
+    wq = _c(wq, np.int8)
+    M, K = c.shape
+    N = wq.shape[0]
+    assert wq.shape == (N, K) and z.shape == (T,)
+    acc = np.empty((M, N), np.int32)
+    if lib().ptqo_int_matmul_asym(_p(c), _p(z), T, _p(wq), M, K, N, _p(acc)):
+        raise OverflowError("accumulator does not fit in int32")
+    return acc
+
+
+def calibrate_asym(xcal, wq, dw):
+    """xcal fp16 [Bc,T,K] -> (s fp32 [K], dx fp32 [T], z int32 [T])."""
+    xcal = _c(xcal, np.float16)
+    Bc, T, K = xcal.shape
+    wq = _c(wq, np.int8)
+    N = wq.shape[0]
+    assert wq.shape == (N, K)
+    dw = _c(dw, np.float32)
+    s = np.empty(K, np.float32)
+    dx = np.empty(T, np.float32)
+    z = np.empty(T, np.int32)
+    lib().ptqo_calibrate_asym(_p(xcal), Bc, T, K, _p(wq), _p(dw), N, _p(s), _p(dx), _p(z))
+    return s, dx, z
+
+
+def linear_forward_asym(x, T, wq, dw, s, dx, z, bias=None, rows=None, taps=False):
+    """Whole asymmetric path on rows [m0, m1): y fp16, or (y, codes uint8, acc int32) with taps."""
+    x = _c(x, np.float16)
+    M, K = x.shape
+    wq = _c(wq, np.int8)
+    N = wq.shape[0]
+    assert wq.shape == (N, K)
+    dw = _c(dw, np.float32)
+    s = _c(s, np.float32)
+    dx = _c(dx, np.float32)
+    z = _c(z, np.int32)
+    assert dw.shape == (N,) and s.shape == (K,) and dx.shape == (T,) and z.shape == (T,)
+    if bias is not None:
+        bias = _c(bias, np.float32)
+    m0, m1 = (0, M) if rows is None else rows
+    R = m1 - m0
+    y = np.empty((R, N), np.float16)
+    c = np.empty((R, K), np.uint8) if taps else None
+    acc = np.empty((R, N), np.int32) if taps else None
+    rc = lib().ptqo_linear_forward_rows_asym(_p(x), m0, m1, K, N, T, _p(wq), _p(dw), _p(s), _p(dx), _p(z),
+                                             _p(bias), _p(y), _p(c), _p(acc))
+    if rc < 0:
+        raise ValueError("K too large for the oracle's row buffer")
+    if rc:
+        raise OverflowError("accumulator does not fit in int32")
+    return (y, c, acc) if taps else y

@@ -24,6 +24,7 @@
 #include <math.h>
 #include <stdint.h>
 #include <stddef.h>
+#include <stdlib.h>
 #include <string.h>
 
 #ifdef _OPENMP
@@ -260,4 +261,143 @@ void ptqo_calibrate(const uint16_t *xcal, int Bc, int T, int K,
             dx[t] = d;
         }
     }
+}
+
+/* ========================================================================= */
+/* Asymmetric PTS: step AND zero offset per token position (Sec. 5.1: "we can  */
+/* allocate the quantization step size and zero offset for each token";       */
+/* quantizer form of Sec. 2.3:                                                */
+/*   X-hat = Delta (clip(round(X / Delta) + eps, 0, 2^b - 1) - eps) ).        */
+/* Reading: the offset eps is an integer z[t] in [0, 255] (the codes must be  */
+/* integers for the integer GEMM), the code is                                */
+/*   c = clip( round((x / s[k]) / dx[t]) + z[t], 0, 255 )        (unsigned)   */
+/* with the same two binary32 divisions and tie rule as the symmetric case,   */
+/* NaN -> z[t] (the value zero), +inf -> 255, -inf -> 0, and the contraction  */
+/* runs over the offset-free integers:                                        */
+/*   acc[m,n] = sum_k (c[m,k] - z[t]) * Wq[n,k].                              */
+/* Dequantization is unchanged.                                               */
+/* Pinned: numpy float32 on all fp16 inputs; z = 128 reproduces the symmetric */
+/* codes; closed form with integer inputs; reconstruction bound; calibration  */
+/* against numpy and the never-clips invariant.                               */
+/* ========================================================================= */
+uint8_t ptqo_quantize_asym_one(uint16_t x_half, float s, float dx, int z)
+{
+    volatile float xf = ptqo_half_to_float(x_half);
+    volatile float u = xf / s;
+    volatile float v = u / dx;
+    double r;
+    if (isnan(v)) return (uint8_t)z;
+    r = (double)nearbyintf(v) + (double)z;      /* exact in binary64, also for infinities */
+    if (r > 255.0) r = 255.0;
+    if (r < 0.0) r = 0.0;
+    return (uint8_t)r;
+}
+
+void ptqo_quantize_asym(const uint16_t *x, long M, int K, int T,
+                        const float *s, const float *dx, const int32_t *z, uint8_t *c)
+{
+    long m;
+#pragma omp parallel for schedule(static)
+    for (m = 0; m < M; ++m) {
+        int t = (int)(m % T);
+        int k;
+        for (k = 0; k < K; ++k)
+            c[m * K + k] = ptqo_quantize_asym_one(x[m * K + k], s[k], dx[t], z[t]);
+    }
+}
+
+int ptqo_int_matmul_asym(const uint8_t *c, const int32_t *z, int T, const int8_t *wq,
+                         long M, int K, int N, int32_t *acc)
+{
+    long m;
+    int overflow = 0;
+#pragma omp parallel for schedule(static) reduction(|:overflow)
+    for (m = 0; m < M; ++m) {
+        int t = (int)(m % T);
+        int n, k;
+        for (n = 0; n < N; ++n) {
+            int64_t sum = 0;
+            for (k = 0; k < K; ++k)
+                sum += ((int64_t)c[m * K + k] - (int64_t)z[t]) * (int64_t)wq[(long)n * K + k];
+            if (sum > INT32_MAX || sum < INT32_MIN) overflow = 1;
+            acc[m * N + n] = (int32_t)sum;
+        }
+    }
+    return overflow;
+}
+
+/* Min-max calibration with zero offset:                                      */
+/*   s[k] as in ptqo_calibrate (Eq. smooth_scale)                             */
+/*   lo[t] = min(0, min_{b,k} x/s),  hi[t] = max(0, max_{b,k} x/s)            */
+/*   dx[t] = max(hi - lo, floor) / 255          (Delta_X of Sec. 2.3)         */
+/*   z[t]  = clip(round(-lo / dx[t]), 0, 255)   (eps_X of Sec. 2.3, rounded)  */
+/* The range always contains zero, so that zero is a code.                    */
+void ptqo_calibrate_asym(const uint16_t *xcal, int Bc, int T, int K,
+                         const int8_t *wq, const float *dw, int N,
+                         float *s, float *dx, int32_t *z)
+{
+    const float floor_ = 1e-5f;
+    float *dx_sym = (float *)malloc(sizeof(float) * (size_t)T);
+    int t;
+    ptqo_calibrate(xcal, Bc, T, K, wq, dw, N, s, dx_sym);    /* s only; the symmetric steps are discarded */
+    free(dx_sym);
+    for (t = 0; t < T; ++t) {
+        float lo = 0.0f, hi = 0.0f;
+        int b, k;
+        for (b = 0; b < Bc; ++b) {
+            long m = (long)b * T + t;
+            for (k = 0; k < K; ++k) {
+                volatile float u = ptqo_half_to_float(xcal[m * K + k]) / s[k];
+                if (u < lo) lo = u;
+                if (u > hi) hi = u;
+            }
+        }
+        {
+            volatile float range = hi - lo;
+            volatile float d;
+            volatile float zr;
+            float r;
+            if (range < floor_) range = floor_;
+            d = range / 255.0f;
+            zr = -lo / d;
+            r = nearbyintf(zr);
+            if (r > 255.0f) r = 255.0f;
+            if (r < 0.0f) r = 0.0f;
+            dx[t] = d;
+            z[t] = (int32_t)r;
+        }
+    }
+}
+
+/* Whole asymmetric path on rows [m0, m1): codes, offset-free accumulators, fp16 output. */
+int ptqo_linear_forward_rows_asym(const uint16_t *x, long m0, long m1, int K, int N, int T,
+                                  const int8_t *wq, const float *dw, const float *s,
+                                  const float *dx, const int32_t *z, const float *bias,
+                                  uint16_t *y, uint8_t *c_out, int32_t *acc_out)
+{
+    long m;
+    int overflow = 0;
+    if (K > PTQO_MAX_K) return -1;
+#pragma omp parallel for schedule(static) reduction(|:overflow)
+    for (m = m0; m < m1; ++m) {
+        int t = (int)(m % T);
+        uint8_t crow[PTQO_MAX_K];
+        int n, k;
+        for (k = 0; k < K; ++k) {
+            crow[k] = ptqo_quantize_asym_one(x[m * K + k], s[k], dx[t], z[t]);
+            if (c_out) c_out[(m - m0) * K + k] = crow[k];
+        }
+        for (n = 0; n < N; ++n) {
+            int64_t sum = 0;
+            double yd;
+            for (k = 0; k < K; ++k)
+                sum += ((int64_t)crow[k] - (int64_t)z[t]) * (int64_t)wq[(long)n * K + k];
+            if (sum > INT32_MAX || sum < INT32_MIN) overflow = 1;
+            if (acc_out) acc_out[(m - m0) * N + n] = (int32_t)sum;
+            yd = (double)(int32_t)sum * (double)dx[t] * (double)dw[n];
+            if (bias) yd += (double)bias[n];
+            y[(m - m0) * N + n] = ptqo_double_to_half(yd);
+        }
+    }
+    return overflow;
 }
