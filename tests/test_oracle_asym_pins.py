@@ -122,6 +122,22 @@ def test_asym_calibration_vs_numpy_and_never_clips():
     assert np.all(err[ok] <= np.broadcast_to(bound, err.shape)[ok])
 
 
+def test_asym_calibration_range_contains_zero_and_degenerate_positions():
+    T, K = 3, 4
+    xcal = np.zeros((2, T, K), np.float16)
+    xcal[:, 0, :] = [[2, 3, 4, 5], [2.5, 3.5, 4.5, 5]]       # all positive: lo is pinned to 0, offset 0
+    xcal[:, 1, :] = [[-2, -3, -4, -5], [-2.5, -3.5, -4.5, -5]]  # all negative: hi is pinned to 0, offset 255
+    wq = np.array([[10, 10, 10, 10]], np.int8)
+    dw = np.array([0.1], F32)                                  # maxW = 1 -> s = sqrt(5)
+    s, dx, z = oracle.calibrate_asym(xcal, wq, dw)
+    s_np, dx_np, z_np = numpy_calibrate_asym(xcal, wq, dw)
+    assert np.array_equal(s, s_np) and np.array_equal(dx, dx_np) and np.array_equal(z, z_np)
+    assert z.tolist() == [0, 255, 0]
+    hi = F32(5) / s[3]
+    assert dx[0] == F32(hi / F32(255)) and dx[1] == dx[0]
+    assert dx[2] == F32(F32(1e-5) / F32(255))                  # dead position: floored range
+
+
 def test_asym_forward_rows_equals_composition():
     spec = wl.configs()[0][0]
     x = wl.activations(spec, wl.ROLE_EVAL, B=2).reshape(-1, spec.K)

@@ -81,7 +81,7 @@ MUTANTS = [
     ("zero offset truncated", "r = nearbyintf(zr);", "r = floorf(zr);",
      [lambda: apins.test_asym_calibration_vs_numpy_and_never_clips()]),
     ("range does not include zero", "float lo = 0.0f, hi = 0.0f;", "float lo = 1e30f, hi = -1e30f;",
-     [lambda: apins.test_asym_calibration_vs_numpy_and_never_clips()]),
+     [lambda: apins.test_asym_calibration_range_contains_zero_and_degenerate_positions()]),
 ]
 
 
