@@ -84,6 +84,24 @@ ptq_status_t ptq_linear_create(ptq_linear_t **out, int K, int N, int T,
                                const float *smooth, const float *act_step,
                                const float *bias, unsigned flags);
 
+/*
+ * Create a layer with ASYMMETRIC per-token-static activations: step and zero offset per token position,
+ * which is what Sec. 5.1 allocates ("step size and zero offset for each token"; quantizer form of
+ * Sec. 2.3 with the offset rounded to an integer):
+ *   Q1  c[m,k]   = clip( rne( (x[m,k] / s[k]) / dx[t] ) + z[t], 0, 255 )           uint8
+ *       (NaN -> z[t], +inf -> 255, -inf -> 0)
+ *   G1  acc[m,n] = sum_k (c[m,k] - z[t]) * Wq[n,k]                                 int32
+ *   E1  as for the symmetric layer
+ *   act_zero   host, [T] int32, zero offsets z[t] in [0,255]
+ * Everything else as ptq_linear_create.  The same forward / quantize / debug entry points serve the
+ * handle; its codes are unsigned bytes.  PTQ_FLAG_FUSED_PROLOGUE and PTQ_FLAG_CTA_PAIR are accepted and
+ * ignored for such a layer (it always runs the quantize kernel and the single-CTA GEMM kernel).
+ */
+ptq_status_t ptq_linear_create_asym(ptq_linear_t **out, int K, int N, int T,
+                                    const int8_t *w_q, const float *w_step,
+                                    const float *smooth, const float *act_step,
+                                    const int32_t *act_zero, const float *bias, unsigned flags);
+
 /* Release the handle and its device memory.  NULL is allowed. */
 void ptq_linear_destroy(ptq_linear_t *h);
 
@@ -189,6 +207,16 @@ ptq_status_t ptq_linear_forward_debug(const ptq_linear_t *h, const void *x_fp16,
 ptq_status_t ptq_calibrate(int K, int N, int T, const void *xcal_fp16, int Bc,
                            const int8_t *w_q, const float *w_step,
                            float *smooth_out, float *act_step_out, void *stream);
+
+/*
+ * Q0 for asymmetric layers: s[k] as in ptq_calibrate; per token position the range [lo, hi] of x/s over
+ * the calibration batch, widened to contain zero; dx[t] = max(hi - lo, 1e-5) / 255 and
+ * z[t] = clip(rne(-lo / dx[t]), 0, 255)  (Delta_X and eps_X of Sec. 2.3 per token position, Sec. 5.1).
+ *   act_zero_out  host, [T] int32
+ */
+ptq_status_t ptq_calibrate_asym(int K, int N, int T, const void *xcal_fp16, int Bc, const int8_t *w_q,
+                                const float *w_step, float *smooth_out, float *act_step_out,
+                                int32_t *act_zero_out, void *stream);
 
 /*
  * Read and clear the handle's device status word.  Synchronises the device.  Returns PTQ_OK, or

@@ -52,6 +52,10 @@ def load_library() -> ctypes.CDLL:
     vp, ci, cu, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_uint, ctypes.c_size_t
     L.ptq_linear_create.restype = ci
     L.ptq_linear_create.argtypes = [ctypes.POINTER(vp), ci, ci, ci, vp, vp, vp, vp, vp, cu]
+    L.ptq_linear_create_asym.restype = ci
+    L.ptq_linear_create_asym.argtypes = [ctypes.POINTER(vp), ci, ci, ci, vp, vp, vp, vp, vp, vp, cu]
+    L.ptq_calibrate_asym.restype = ci
+    L.ptq_calibrate_asym.argtypes = [ci, ci, ci, vp, ci, vp, vp, vp, vp, vp, vp]
     L.ptq_linear_destroy.restype = None
     L.ptq_linear_destroy.argtypes = [vp]
     L.ptq_linear_workspace_bytes.restype = sz
@@ -118,7 +122,7 @@ def kernel_launch_count() -> int:
 class PtqLinear:
     """One PTS W8A8 linear layer on the current CUDA device (``ptq_linear_create``)."""
 
-    def __init__(self, w_q, w_step, smooth, act_step, bias=None, flags: int = 0):
+    def __init__(self, w_q, w_step, smooth, act_step, bias=None, flags: int = 0, act_zero=None):
         L = load_library()
         w_q = _host(w_q, np.int8)
         if w_q.ndim != 2:
@@ -130,8 +134,14 @@ class PtqLinear:
         smooth = _host(smooth, np.float32, (self.K,))
         bias = _host(bias, np.float32, (self.N,))
         h = ctypes.c_void_p()
-        _check(L.ptq_linear_create(ctypes.byref(h), self.K, self.N, self.T, _hp(w_q), _hp(w_step),
-                                   _hp(smooth), _hp(act_step), _hp(bias), flags))
+        self.asym = act_zero is not None
+        if self.asym:                                            # ``ptq_linear_create_asym``: unsigned codes
+            act_zero = _host(act_zero, np.int32, (self.T,))
+            _check(L.ptq_linear_create_asym(ctypes.byref(h), self.K, self.N, self.T, _hp(w_q), _hp(w_step),
+                                            _hp(smooth), _hp(act_step), _hp(act_zero), _hp(bias), flags))
+        else:
+            _check(L.ptq_linear_create(ctypes.byref(h), self.K, self.N, self.T, _hp(w_q), _hp(w_step),
+                                       _hp(smooth), _hp(act_step), _hp(bias), flags))
         self._h = h
         self._L = L
 
@@ -202,7 +212,7 @@ class PtqLinear:
         import torch
         B = self._batch(x)
         if q is None:
-            q = torch.empty((B, self.T, self.K), dtype=torch.int8, device=x.device)
+            q = torch.empty((B, self.T, self.K), dtype=torch.uint8 if self.asym else torch.int8, device=x.device)
         _check(self._L.ptq_quantize(self._h, x.data_ptr(), B, q.data_ptr(), _stream_ptr(stream)))
         return q
 
@@ -227,7 +237,8 @@ class PtqLinear:
         B = self._batch(x)
         dev = x.device
         y = torch.empty((B, self.T, self.N), dtype=torch.float16, device=dev)
-        q = torch.empty((B, self.T, self.K), dtype=torch.int8, device=dev) if want_q else None
+        q = torch.empty((B, self.T, self.K), dtype=torch.uint8 if self.asym else torch.int8,
+                        device=dev) if want_q else None
         acc = torch.empty((B, self.T, self.N), dtype=torch.int32, device=dev) if want_acc else None
         need = self.workspace_bytes(B, 0)
         ws = torch.empty(need, dtype=torch.uint8, device=dev)
@@ -256,3 +267,23 @@ def calibrate(xcal, w_q, w_step, stream=None):
     _check(L.ptq_calibrate(K, N, T, xcal.data_ptr(), Bc, _hp(w_q), _hp(w_step), _hp(s), _hp(dx),
                            _stream_ptr(stream)))
     return s, dx
+
+
+def calibrate_asym(xcal, w_q, w_step, stream=None):
+    """``ptq_calibrate_asym``: device fp16 [Bc,T,K] -> (s fp32 [K], dx fp32 [T], z int32 [T])."""
+    import torch
+    L = load_library()
+    if xcal.dtype != torch.float16 or not xcal.is_cuda or not xcal.is_contiguous() or xcal.dim() != 3:
+        raise ValueError("xcal must be a contiguous CUDA float16 tensor [Bc,T,K]")
+    Bc, T, K = (int(v) for v in xcal.shape)
+    w_q = _host(w_q, np.int8)
+    N = int(w_q.shape[0])
+    if w_q.shape != (N, K):
+        raise ValueError("w_q must be [N,K]")
+    w_step = _host(w_step, np.float32, (N,))
+    s = np.empty(K, np.float32)
+    dx = np.empty(T, np.float32)
+    z = np.empty(T, np.int32)
+    _check(L.ptq_calibrate_asym(K, N, T, xcal.data_ptr(), Bc, _hp(w_q), _hp(w_step), _hp(s), _hp(dx), _hp(z),
+                                _stream_ptr(stream)))
+    return s, dx, z

@@ -113,6 +113,9 @@ struct ptq_linear {
     float *d_s = nullptr, *d_rs = nullptr;               // [round_up(K,16)]
     float *d_dx = nullptr, *d_rdx = nullptr;             // [T]
     float2 *d_dx2 = nullptr;                             // [T] {dx, 1/dx}
+    int *d_zp = nullptr;                                 // [T] zero offsets (asymmetric layers only)
+    int *d_wsum = nullptr;                               // row sums of Wq, padded like d_dw (asymmetric only)
+    bool asym = false;
     unsigned *d_status = nullptr;
     CUtensorMap tmW;
     CUtensorMap tmWh;          // same weights, box of BN/2 rows: the half tile one CTA of a pair loads
@@ -195,6 +198,7 @@ ptq_status_t launch_quantize(const ptq_linear *h, const void *x, long long M, vo
     p.dx = h->d_dx;
     p.rdx = h->d_rdx;
     p.dx2 = h->d_dx2;
+    p.zp = h->d_zp;
     p.M = M;
     p.K = h->K;
     p.T = h->T;
@@ -221,7 +225,12 @@ ptq_status_t launch_quantize(const ptq_linear *h, const void *x, long long M, vo
     p.imgs_per_iter = static_cast<int>(S);
     if (vec) {
         const int grid = static_cast<int>(S * cpi / 256);
-        if (h->fast_div)
+        if (h->asym) {
+            if (h->fast_div)
+                ptq::ptq_quantize_vec8_kernel<true, true><<<grid, 256, 0, stream>>>(p);
+            else
+                ptq::ptq_quantize_vec8_kernel<false, true><<<grid, 256, 0, stream>>>(p);
+        } else if (h->fast_div)
             ptq::ptq_quantize_vec8_kernel<true><<<grid, 256, 0, stream>>>(p);
         else
             ptq::ptq_quantize_vec8_kernel<false><<<grid, 256, 0, stream>>>(p);
@@ -230,7 +239,12 @@ ptq_status_t launch_quantize(const ptq_linear *h, const void *x, long long M, vo
         const long long cap = static_cast<long long>(h->num_sms) * 8;
         if (want > cap) want = cap;
         if (want < 1) want = 1;
-        if (h->fast_div)
+        if (h->asym) {
+            if (h->fast_div)
+                ptq::ptq_quantize_scalar_kernel<true, true><<<static_cast<int>(want), 256, 0, stream>>>(p);
+            else
+                ptq::ptq_quantize_scalar_kernel<false, true><<<static_cast<int>(want), 256, 0, stream>>>(p);
+        } else if (h->fast_div)
             ptq::ptq_quantize_scalar_kernel<true><<<static_cast<int>(want), 256, 0, stream>>>(p);
         else
             ptq::ptq_quantize_scalar_kernel<false><<<static_cast<int>(want), 256, 0, stream>>>(p);
@@ -286,6 +300,8 @@ ptq_status_t launch_gemm(const ptq_linear *h, const void *codes, long long M, vo
     p.use_tma_store = tma_store ? 1 : 0;
     p.y_vec2 = (h->N % 2 == 0 && reinterpret_cast<uintptr_t>(y) % 4 == 0) ? 1 : 0;
     p.y_vec8 = 0;   // this kernel always has a staging buffer; 16-byte alignment means TMA stores
+    p.zp = h->d_zp;
+    p.wsum = h->d_wsum;
 
     const long long pair_tiles = static_cast<long long>((p.m_tiles + 1) / 2) * p.n_tiles;
     if (want_pair && h->max_pairs > 0 && pair_tiles >= h->max_pairs) {
@@ -406,6 +422,8 @@ ptq_status_t launch_astat(const ptq_linear *h, const void *src, bool quantize, l
     p.use_tma_store = tma_store ? 1 : 0;
     p.y_vec2 = (h->N % 2 == 0 && reinterpret_cast<uintptr_t>(y) % 4 == 0) ? 1 : 0;
     p.y_vec8 = (aligned && !tma_store) ? 1 : 0;
+    p.zp = nullptr;
+    p.wsum = nullptr;
     fp.x = static_cast<const __half *>(quantize ? src : nullptr);
     fp.s = h->d_s;
     fp.rs = h->d_rs;
@@ -508,12 +526,15 @@ void ptq_linear_destroy(ptq_linear_t *h)
     cudaFree(h->d_dx);
     cudaFree(h->d_rdx);
     cudaFree(h->d_dx2);
+    cudaFree(h->d_zp);
+    cudaFree(h->d_wsum);
     cudaFree(h->d_status);
     delete h;
 }
 
-ptq_status_t ptq_linear_create(ptq_linear_t **out, int K, int N, int T, const int8_t *w_q, const float *w_step,
-                               const float *smooth, const float *act_step, const float *bias, unsigned flags)
+static ptq_status_t create_impl(ptq_linear_t **out, int K, int N, int T, const int8_t *w_q, const float *w_step,
+                                const float *smooth, const float *act_step, const int32_t *act_zero,
+                                const float *bias, unsigned flags)
 {
     if (!out) return fail(PTQ_ERR_NULL, "out must not be NULL");
     *out = nullptr;
@@ -541,6 +562,9 @@ ptq_status_t ptq_linear_create(ptq_linear_t **out, int K, int N, int T, const in
             return fail(PTQ_ERR_VALUE, "w_step[%d] = %g must be finite and > 0", n, w_step[n]);
         if (bias && !std::isfinite(bias[n])) return fail(PTQ_ERR_VALUE, "bias[%d] is not finite", n);
     }
+    for (int t = 0; act_zero && t < T; ++t)
+        if (act_zero[t] < 0 || act_zero[t] > 255)
+            return fail(PTQ_ERR_VALUE, "act_zero[%d] = %d is outside [0,255]", t, act_zero[t]);
     for (long long i = 0; i < static_cast<long long>(N) * K; ++i)
         if (w_q[i] == -128)
             return fail(PTQ_ERR_VALUE, "w_q[%lld] = -128 is outside the symmetric range [-127,127]", i);
@@ -570,7 +594,9 @@ ptq_status_t ptq_linear_create(ptq_linear_t **out, int K, int N, int T, const in
     h->k_blocks = (K + ptq::kBK - 1) / ptq::kBK;
     h->last_mmas = (K - (h->k_blocks - 1) * ptq::kBK + 31) / 32;
 
+    h->asym = act_zero != nullptr;
     choose_astat(h);
+    if (h->asym) h->as_ok = false;          // asymmetric layers run the quantize kernel + single-CTA GEMM kernel only
     int Npad = h->n_tiles * h->BN;
     if (h->as_ok && h->as_n_tiles * h->as_BN > Npad) Npad = h->as_n_tiles * h->as_BN;
     const int Nvec = round_up(Npad, 64) + 64;
@@ -600,6 +626,16 @@ ptq_status_t ptq_linear_create(ptq_linear_t **out, int K, int N, int T, const in
         if ((st = upload(reinterpret_cast<void **>(&h->d_rdx), rdx.data(), sizeof(float) * T, sizeof(float) * T)) != PTQ_OK) break;
         if ((st = upload(reinterpret_cast<void **>(&h->d_dx2), dx2.data(), sizeof(float) * 2 * T, sizeof(float) * 2 * T)) != PTQ_OK) break;
         if ((st = upload(reinterpret_cast<void **>(&h->d_status), nullptr, 0, sizeof(unsigned))) != PTQ_OK) break;
+        if (h->asym) {
+            std::vector<int> wsum(Nvec, 0);
+            for (int n = 0; n < N; ++n) {
+                int acc = 0;
+                for (int k = 0; k < K; ++k) acc += w_q[static_cast<size_t>(n) * K + k];
+                wsum[n] = acc;
+            }
+            if ((st = upload(reinterpret_cast<void **>(&h->d_zp), act_zero, sizeof(int) * T, sizeof(int) * T)) != PTQ_OK) break;
+            if ((st = upload(reinterpret_cast<void **>(&h->d_wsum), wsum.data(), sizeof(int) * Nvec, sizeof(int) * Nvec)) != PTQ_OK) break;
+        }
         st = make_map_2d(&h->tmW, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, h->d_w, static_cast<unsigned long long>(K),
                          static_cast<unsigned long long>(Npad), static_cast<unsigned long long>(h->Kpad), ptq::kBK,
                          static_cast<unsigned>(h->BN));
@@ -608,7 +644,7 @@ ptq_status_t ptq_linear_create(ptq_linear_t **out, int K, int N, int T, const in
                          static_cast<unsigned long long>(Npad), static_cast<unsigned long long>(h->Kpad), ptq::kBK,
                          static_cast<unsigned>(h->BN / 2));
         if (st != PTQ_OK) break;
-        h->max_pairs = query_max_pairs();
+        h->max_pairs = h->asym ? 0 : query_max_pairs();
         if (h->as_ok)
             st = make_map_2d(&h->tmWas, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, h->d_w, static_cast<unsigned long long>(K),
                              static_cast<unsigned long long>(Npad), static_cast<unsigned long long>(h->Kpad),
@@ -625,6 +661,21 @@ ptq_status_t ptq_linear_create(ptq_linear_t **out, int K, int N, int T, const in
     }
     *out = h;
     return PTQ_OK;
+}
+
+ptq_status_t ptq_linear_create(ptq_linear_t **out, int K, int N, int T, const int8_t *w_q, const float *w_step,
+                               const float *smooth, const float *act_step, const float *bias, unsigned flags)
+{
+    return create_impl(out, K, N, T, w_q, w_step, smooth, act_step, nullptr, bias, flags);
+}
+
+ptq_status_t ptq_linear_create_asym(ptq_linear_t **out, int K, int N, int T, const int8_t *w_q, const float *w_step,
+                                    const float *smooth, const float *act_step, const int32_t *act_zero,
+                                    const float *bias, unsigned flags)
+{
+    if (out) *out = nullptr;
+    if (!act_zero) return fail(PTQ_ERR_NULL, "act_zero must not be NULL");
+    return create_impl(out, K, N, T, w_q, w_step, smooth, act_step, act_zero, bias, flags);
 }
 
 size_t ptq_linear_workspace_bytes(const ptq_linear_t *h, int B, unsigned flags)
@@ -654,9 +705,10 @@ int ptq_linear_describe(const ptq_linear_t *h, char *buf, int buf_bytes)
     if (!h) return 0;
     char tmp[512];
     const int n = snprintf(tmp, sizeof(tmp),
-                           "K=%d N=%d T=%d Kpad=%d | quantize: %s | gemm: BN=%d n_tiles=%d k_blocks=%d "
+                           "K=%d N=%d T=%d Kpad=%d%s | quantize: %s | gemm: BN=%d n_tiles=%d k_blocks=%d "
                            "pair_clusters=%d | fused: %s BN=%d n_tiles=%d w_stages=%d staging=%d smem=%d",
-                           h->K, h->N, h->T, h->Kpad, h->fast_div ? "screened reciprocal route" : "IEEE division",
+                           h->K, h->N, h->T, h->Kpad, h->asym ? " asymmetric" : "",
+                           h->fast_div ? "screened reciprocal route" : "IEEE division",
                            h->BN, h->n_tiles, h->k_blocks, h->max_pairs,
                            (h->as_ok && h->K % 16 == 0) ? "yes" : "no", h->as_BN, h->as_n_tiles, h->as_w_stages,
                            h->as_staging, h->as_smem);
@@ -756,8 +808,9 @@ ptq_status_t ptq_linear_device_status(const ptq_linear_t *h)
     return PTQ_OK;
 }
 
-ptq_status_t ptq_calibrate(int K, int N, int T, const void *xcal_fp16, int Bc, const int8_t *w_q,
-                           const float *w_step, float *smooth_out, float *act_step_out, void *stream)
+static ptq_status_t calibrate_impl(int K, int N, int T, const void *xcal_fp16, int Bc, const int8_t *w_q,
+                                   const float *w_step, float *smooth_out, float *act_step_out,
+                                   int32_t *act_zero_out, void *stream)
 {
     if (!xcal_fp16 || !w_q || !w_step || !smooth_out || !act_step_out)
         return fail(PTQ_ERR_NULL, "calibrate: pointers must not be NULL");
@@ -770,17 +823,17 @@ ptq_status_t ptq_calibrate(int K, int N, int T, const void *xcal_fp16, int Bc, c
     PTQ_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
     const long long M = static_cast<long long>(Bc) * T;
 
-    unsigned *d_bits = nullptr;   // [K] maxX bits, then [T] mu bits
-    float *d_out = nullptr;       // [K] s, then [T] dx
+    unsigned *d_bits = nullptr;   // [K] maxX bits, then [T] mu (or hi) bits, then [T] -lo bits
+    float *d_out = nullptr;       // [K] s, then [T] dx, then [T] z (int)
     float *d_dw = nullptr;
     int8_t *d_w = nullptr;
     ptq_status_t st = PTQ_OK;
     auto body = [&]() -> ptq_status_t {
-        PTQ_CUDA(cudaMalloc(reinterpret_cast<void **>(&d_bits), sizeof(unsigned) * (K + T)));
-        PTQ_CUDA(cudaMalloc(reinterpret_cast<void **>(&d_out), sizeof(float) * (K + T)));
+        PTQ_CUDA(cudaMalloc(reinterpret_cast<void **>(&d_bits), sizeof(unsigned) * (K + 2 * T)));
+        PTQ_CUDA(cudaMalloc(reinterpret_cast<void **>(&d_out), sizeof(float) * (K + 2 * T)));
         PTQ_CUDA(cudaMalloc(reinterpret_cast<void **>(&d_dw), sizeof(float) * N));
         PTQ_CUDA(cudaMalloc(reinterpret_cast<void **>(&d_w), static_cast<size_t>(N) * K));
-        PTQ_CUDA(cudaMemsetAsync(d_bits, 0, sizeof(unsigned) * (K + T), s));
+        PTQ_CUDA(cudaMemsetAsync(d_bits, 0, sizeof(unsigned) * (K + 2 * T), s));
         PTQ_CUDA(cudaMemcpyAsync(d_dw, w_step, sizeof(float) * N, cudaMemcpyHostToDevice, s));
         PTQ_CUDA(cudaMemcpyAsync(d_w, w_q, static_cast<size_t>(N) * K, cudaMemcpyHostToDevice, s));
         const __half *x = static_cast<const __half *>(xcal_fp16);
@@ -789,12 +842,20 @@ ptq_status_t ptq_calibrate(int K, int N, int T, const void *xcal_fp16, int Bc, c
         const int grid = static_cast<int>(want < 1 ? 1 : want);
         ptq::ptq_calib_colmax_kernel<<<grid, 256, 0, s>>>(x, M, K, d_bits);
         ptq::ptq_calib_smooth_kernel<<<(K + 127) / 128, 128, 0, s>>>(d_bits, d_w, d_dw, N, K, d_out);
-        ptq::ptq_calib_rowmax_kernel<<<grid, 256, 0, s>>>(x, M, K, T, d_out, d_bits + K);
-        ptq::ptq_calib_step_kernel<<<(T + 127) / 128, 128, 0, s>>>(d_bits + K, T, d_out + K);
+        if (act_zero_out) {
+            ptq::ptq_calib_rowrange_kernel<<<grid, 256, 0, s>>>(x, M, K, T, d_out, d_bits + K, d_bits + K + T);
+            ptq::ptq_calib_step_asym_kernel<<<(T + 127) / 128, 128, 0, s>>>(d_bits + K, d_bits + K + T, T, d_out + K,
+                                                                           reinterpret_cast<int *>(d_out + K + T));
+        } else {
+            ptq::ptq_calib_rowmax_kernel<<<grid, 256, 0, s>>>(x, M, K, T, d_out, d_bits + K);
+            ptq::ptq_calib_step_kernel<<<(T + 127) / 128, 128, 0, s>>>(d_bits + K, T, d_out + K);
+        }
         g_launches.fetch_add(4, std::memory_order_relaxed);
         PTQ_CUDA(cudaGetLastError());
         PTQ_CUDA(cudaMemcpyAsync(smooth_out, d_out, sizeof(float) * K, cudaMemcpyDeviceToHost, s));
         PTQ_CUDA(cudaMemcpyAsync(act_step_out, d_out + K, sizeof(float) * T, cudaMemcpyDeviceToHost, s));
+        if (act_zero_out)
+            PTQ_CUDA(cudaMemcpyAsync(act_zero_out, d_out + K + T, sizeof(int32_t) * T, cudaMemcpyDeviceToHost, s));
         PTQ_CUDA(cudaStreamSynchronize(s));
         return PTQ_OK;
     };
@@ -804,6 +865,20 @@ ptq_status_t ptq_calibrate(int K, int N, int T, const void *xcal_fp16, int Bc, c
     cudaFree(d_dw);
     cudaFree(d_w);
     return st;
+}
+
+ptq_status_t ptq_calibrate(int K, int N, int T, const void *xcal_fp16, int Bc, const int8_t *w_q,
+                           const float *w_step, float *smooth_out, float *act_step_out, void *stream)
+{
+    return calibrate_impl(K, N, T, xcal_fp16, Bc, w_q, w_step, smooth_out, act_step_out, nullptr, stream);
+}
+
+ptq_status_t ptq_calibrate_asym(int K, int N, int T, const void *xcal_fp16, int Bc, const int8_t *w_q,
+                                const float *w_step, float *smooth_out, float *act_step_out,
+                                int32_t *act_zero_out, void *stream)
+{
+    if (!act_zero_out) return fail(PTQ_ERR_NULL, "calibrate: pointers must not be NULL");
+    return calibrate_impl(K, N, T, xcal_fp16, Bc, w_q, w_step, smooth_out, act_step_out, act_zero_out, stream);
 }
 
 }  // extern "C"

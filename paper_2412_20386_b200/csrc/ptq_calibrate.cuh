@@ -96,4 +96,46 @@ __global__ void __launch_bounds__(128) ptq_calib_step_kernel(const unsigned *mu_
     dx[t] = __fdiv_rn(fmaxf(__uint_as_float(mu_bits[t]), kCalibFloor), 127.0f);
 }
 
+// --- asymmetric variant: per-token-position range [lo, hi] of x/s, always containing zero ----------
+//   hi[t] = max(0, max x/s),  nlo[t] = max(0, max -(x/s))   (both non-negative: atomicMax on the bits)
+//   dx[t] = max(hi + nlo, 1e-5) / 255,   z[t] = clip(rne(nlo / dx[t]), 0, 255)
+__global__ void __launch_bounds__(256) ptq_calib_rowrange_kernel(const __half *x, long long M, int K, int T,
+                                                                 const float *s, unsigned *hi_bits,
+                                                                 unsigned *nlo_bits)
+{
+    const int lane = threadIdx.x & 31;
+    const int warps_per_block = blockDim.x >> 5;
+    const long long warp = static_cast<long long>(blockIdx.x) * warps_per_block + (threadIdx.x >> 5);
+    const long long nwarps = static_cast<long long>(gridDim.x) * warps_per_block;
+    for (long long m = warp; m < M; m += nwarps) {
+        const __half *row = x + m * K;
+        float hi = 0.0f, nlo = 0.0f;
+        for (int k = lane; k < K; k += 32) {
+            const float u = __fdiv_rn(__half2float(row[k]), __ldg(s + k));
+            hi = fmaxf(hi, u);          // fmaxf drops NaN
+            nlo = fmaxf(nlo, -u);
+        }
+        hi = warp_max(hi);
+        nlo = warp_max(nlo);
+        if (lane == 0) {
+            const int t = static_cast<int>(m % T);
+            if (hi > 0.0f) atomicMax(hi_bits + t, __float_as_uint(hi));
+            if (nlo > 0.0f) atomicMax(nlo_bits + t, __float_as_uint(nlo));
+        }
+    }
+}
+
+__global__ void __launch_bounds__(128) ptq_calib_step_asym_kernel(const unsigned *hi_bits, const unsigned *nlo_bits,
+                                                                  int T, float *dx, int *z)
+{
+    const int t = blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= T) return;
+    const float hi = __uint_as_float(hi_bits[t]), nlo = __uint_as_float(nlo_bits[t]);
+    const float range = fmaxf(__fadd_rn(hi, nlo), kCalibFloor);      // hi - lo with lo = -nlo
+    const float d = __fdiv_rn(range, 255.0f);
+    const float zr = rintf(__fdiv_rn(nlo, d));                        // -lo / d, ties to even
+    dx[t] = d;
+    z[t] = static_cast<int>(fminf(fmaxf(zr, 0.0f), 255.0f));
+}
+
 }  // namespace ptq

@@ -59,6 +59,11 @@ struct GemmParams {
     int use_tma_store; // y is written by TMA (needs N % 8 == 0 and a 16-byte aligned y)
     int y_vec2;        // plain-store path may use 4-byte stores (N even, y 4-byte aligned)
     int y_vec8;        // plain-store path may use 16-byte stores (N % 8 == 0, y 16-byte aligned)
+    // Asymmetric layers (zero offset per token position): the codes are unsigned, the tensor core
+    // accumulates sum_k c * Wq, and the epilogue subtracts z[t] * sum_k Wq[n,k] to obtain the offset-free
+    // accumulator sum_k (c - z[t]) * Wq[n,k] exactly (all int32).  nullptr for symmetric layers.
+    const int *zp;     // [T]
+    const int *wsum;   // [>= n_tiles*BN + 64] row sums of Wq, zero padded
 };
 
 // --- epilogue helpers -------------------------------------------------------------------------
@@ -162,7 +167,7 @@ __device__ __forceinline__ void store_acc32(const uint32_t (&v)[32], int32_t *ar
 template <bool kDebugAcc, bool kLowReg = false>
 __device__ __forceinline__ uint32_t epilogue_tile(const GemmParams &p, const CUtensorMap *tmY, uint32_t tmem_row,
                                                   long long m_row0, int n0, float dxr, uint32_t staging,
-                                                  uint32_t nboxes, int lane, int col_half)
+                                                  uint32_t nboxes, int lane, int col_half, int zr = 0)
 {
     const long long m = m_row0 + lane;
     const bool row_ok = m < p.M;
@@ -180,6 +185,17 @@ __device__ __forceinline__ uint32_t epilogue_tile(const GemmParams &p, const CUt
                 tmem_ld_wait();
             }
             const int n_half = n_first + 32 * half;
+            if (p.zp != nullptr) {
+                // offset-free accumulator: acc - z[t] * sum_k Wq[n,k]
+#pragma unroll
+                for (int i4 = 0; i4 < 8; ++i4) {
+                    const int4 ws = __ldg(reinterpret_cast<const int4 *>(p.wsum + n_half) + i4);
+                    v[4 * i4 + 0] -= static_cast<uint32_t>(zr * ws.x);
+                    v[4 * i4 + 1] -= static_cast<uint32_t>(zr * ws.y);
+                    v[4 * i4 + 2] -= static_cast<uint32_t>(zr * ws.z);
+                    v[4 * i4 + 3] -= static_cast<uint32_t>(zr * ws.w);
+                }
+            }
             if (kDebugAcc) {
                 if (p.acc_out != nullptr && row_ok) store_acc32(v, p.acc_out + m * p.N, n_half, p.N);
             }
@@ -295,7 +311,7 @@ ptq_gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            const uint32_t idesc = make_idesc_s8(kBM, p.BN);
+            const uint32_t idesc = make_idesc_s8(kBM, p.BN, p.zp != nullptr);   // unsigned codes on asymmetric layers
             uint32_t stage = 0, phase = 0, buf = 0, bphase = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
@@ -337,13 +353,16 @@ ptq_gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             const int n_tile = tile - m_tile * p.n_tiles;
             const long long m_row0 = static_cast<long long>(m_tile) * kBM + quarter * 32;
             const long long m = m_row0 + lane;
-            const float dxr = (m < p.M) ? __ldg(p.dx + static_cast<int>(m % p.T)) : 0.0f;
+            const int t_row = (m < p.M) ? static_cast<int>(m % p.T) : 0;
+            const float dxr = (m < p.M) ? __ldg(p.dx + t_row) : 0.0f;
+            const int zr = (p.zp != nullptr) ? __ldg(p.zp + t_row) : 0;
             bool got = mbar_wait(tfull_bar(buf), bphase, abort_flag, p.status);
             got = __all_sync(0xffffffffu, got);
             if (!got) break;
             tc_fence_after_sync();
             const uint32_t tmem_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * kMaxBN;
-            nboxes = epilogue_tile<kDebugAcc>(p, &tmY, tmem_row, m_row0, n_tile * p.BN, dxr, staging, nboxes, lane, col_half);
+            nboxes = epilogue_tile<kDebugAcc>(p, &tmY, tmem_row, m_row0, n_tile * p.BN, dxr, staging, nboxes, lane, col_half,
+                                              zr);
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(tempty_bar(buf));

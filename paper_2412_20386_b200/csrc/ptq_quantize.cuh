@@ -35,17 +35,36 @@ __device__ __forceinline__ int f32_to_code(float v)
     return r;
 }
 
-// One element, IEEE divisions (any positive finite s, dx; also the path for inf/NaN inputs).
-__device__ __forceinline__ int quantize_ieee(float xf, float s, float dx)
+// Asymmetric code (zero offset z in [0,255] per token position): clip(rne(v) + z, 0, 255).
+// The offset is added to the rounded INTEGER (adding it in binary32 before rounding would erase ties);
+// cvt.rni.sat.s16.f32 keeps the intermediate inside +-32768 so the addition cannot overflow, and maps
+// NaN to 0, i.e. to the code z.
+__device__ __forceinline__ int f32_to_code_asym(float v, int z)
 {
-    return f32_to_code(__fdiv_rn(__fdiv_rn(xf, s), dx));
+    short r;
+    asm("cvt.rni.sat.s16.f32 %0, %1;" : "=h"(r) : "f"(v));
+    return min(max(static_cast<int>(r) + z, 0), 255);
+}
+
+template <bool kAsym>
+__device__ __forceinline__ int code_of(float v, int z)
+{
+    return kAsym ? f32_to_code_asym(v, z) : f32_to_code(v);
+}
+
+// One element, IEEE divisions (any positive finite s, dx; also the path for inf/NaN inputs).
+template <bool kAsym = false>
+__device__ __forceinline__ int quantize_ieee(float xf, float s, float dx, int z = 0)
+{
+    return code_of<kAsym>(__fdiv_rn(__fdiv_rn(xf, s), dx), z);
 }
 
 // One element through the reciprocal route (finite xf, scales inside the safe range).
-__device__ __forceinline__ int quantize_fast(float xf, float s, float rs, float dx, float rdx)
+template <bool kAsym = false>
+__device__ __forceinline__ int quantize_fast(float xf, float s, float rs, float dx, float rdx, int z = 0)
 {
     const float u = div_rn_by_reciprocal(xf, s, rs);
-    return f32_to_code(div_rn_by_reciprocal(u, dx, rdx));
+    return code_of<kAsym>(div_rn_by_reciprocal(u, dx, rdx), z);
 }
 
 __device__ __forceinline__ uint32_t pack4(int a, int b, int c, int d)
@@ -61,6 +80,9 @@ __device__ __forceinline__ uint32_t pack4(int a, int b, int c, int d)
 // below 4.6e-5 for |v| <= 127.5, the largest magnitude at which a rounding tie still changes the
 // clamped code.  If v' is farther than 6e-5 from every half-integer, rint(v') = rint(v).
 constexpr float kScreenThreshold = 0.49994f;
+// Asymmetric codes: rint(v) ranges over [-255, 255] before the offset, so ties matter up to |v| = 255.5,
+// where six roundings amount to 9.2e-5; the band is widened to 1.2e-4 accordingly.
+constexpr float kScreenThresholdAsym = 0.49988f;
 constexpr float kRoundMagic = 12582912.0f;   // 1.5 * 2^23: (v + magic) - magic = rint(v) for |v| < 2^22
 
 // |v - rint(v)| for |v| < 2^22; NaN for NaN and infinite v; meaningless (but finite or NaN) beyond.
@@ -78,8 +100,11 @@ __device__ __forceinline__ float dist_to_integer(float v)
 // infinities saturate on both routes, so whether such values pass the test or not only costs time:
 // the final codes are always those of the definition.
 // Valid only when every scale lies in [2^-30, 2^30] (no under/overflow in c or x * c).
+// kAsym: the codes are clip(rint(v') + z, 0, 255); ties of v' are still the only place where v' and v
+// can disagree, with the wider band of kScreenThresholdAsym.
+template <bool kAsym = false>
 __device__ __forceinline__ bool quantize8_screen(uint32_t x0, uint32_t x1, uint32_t x2, uint32_t x3,
-                                                 const float (&c8)[8], uint32_t &lo, uint32_t &hi)
+                                                 const float (&c8)[8], uint32_t &lo, uint32_t &hi, int z = 0)
 {
     const uint32_t xw[4] = {x0, x1, x2, x3};
     int c[8];
@@ -91,20 +116,21 @@ __device__ __forceinline__ bool quantize8_screen(uint32_t x0, uint32_t x1, uint3
         const float2 f = __half22float2(h);
         const float v0 = __fmul_rn(f.x, c8[2 * i]);
         const float v1 = __fmul_rn(f.y, c8[2 * i + 1]);
-        c[2 * i] = f32_to_code(v0);
-        c[2 * i + 1] = f32_to_code(v1);
+        c[2 * i] = code_of<kAsym>(v0, z);
+        c[2 * i + 1] = code_of<kAsym>(v1, z);
         worst = fmaxf(worst, fmaxf(dist_to_integer(v0), dist_to_integer(v1)));
     }
     lo = pack4(c[0], c[1], c[2], c[3]);
     hi = pack4(c[4], c[5], c[6], c[7]);
-    return worst > kScreenThreshold;
+    return worst > (kAsym ? kScreenThresholdAsym : kScreenThreshold);
 }
 
 // Exact route for the same 8 channels: two correctly rounded divisions per element.  s8 / rs8 point
 // at the channels' s and RN(1/s) in global memory.
-template <bool kFast>
+template <bool kFast, bool kAsym = false>
 __device__ __noinline__ void quantize8_exact(uint32_t x0, uint32_t x1, uint32_t x2, uint32_t x3, const float *s8,
-                                             const float *rs8, float dx, float rdx, uint32_t &lo, uint32_t &hi)
+                                             const float *rs8, float dx, float rdx, uint32_t &lo, uint32_t &hi,
+                                             int z = 0)
 {
     const uint32_t xw[4] = {x0, x1, x2, x3};
     int c[8];
@@ -114,9 +140,9 @@ __device__ __noinline__ void quantize8_exact(uint32_t x0, uint32_t x1, uint32_t 
         const float f = __half2float(hv);
         const float sv = __ldg(s8 + i);
         if (kFast && fabsf(f) <= 65504.0f)
-            c[i] = quantize_fast(f, sv, __ldg(rs8 + i), dx, rdx);
+            c[i] = quantize_fast<kAsym>(f, sv, __ldg(rs8 + i), dx, rdx, z);
         else
-            c[i] = quantize_ieee(f, sv, dx);
+            c[i] = quantize_ieee<kAsym>(f, sv, dx, z);
     }
     lo = pack4(c[0], c[1], c[2], c[3]);
     hi = pack4(c[4], c[5], c[6], c[7]);
@@ -130,6 +156,7 @@ struct QuantParams {
     const float *dx;     // [T]
     const float *rdx;    // [T]  RN(1/dx)
     const float2 *dx2;   // [T]  {dx, RN(1/dx)} interleaved (one 8-byte load)
+    const int *zp;       // [T]  zero offsets (asymmetric layers), else nullptr
     long long M;
     int K;
     int T;
@@ -156,7 +183,7 @@ constexpr int kQuantImgsPerTrip = PTQ_QUANT_IMGS_PER_TRIP; // 16-byte loads per 
 // in registers, and the per-element work is convert, multiply, round, tie test.  Consecutive lanes
 // take consecutive chunks, so warp-wide accesses are contiguous 512-byte loads and 256-byte stores.
 // Each trip converts kQuantImgsPerTrip chunks and issues the next trip's loads first.
-template <bool kFast>
+template <bool kFast, bool kAsym = false>
 __global__ void __launch_bounds__(256, kQuantCtasPerSm) ptq_quantize_vec8_kernel(QuantParams p)
 {
     constexpr int U = kQuantImgsPerTrip;
@@ -170,6 +197,7 @@ __global__ void __launch_bounds__(256, kQuantCtasPerSm) ptq_quantize_vec8_kernel
     const int S = p.imgs_per_iter;
 
     const float2 d = __ldg(p.dx2 + t);
+    const int z = kAsym ? __ldg(p.zp + t) : 0;
     const float *s8 = p.s + kc * 8;          // read only on the exact route
     const float *rs8 = p.rs + kc * 8;
     float c8[8];
@@ -202,8 +230,9 @@ __global__ void __launch_bounds__(256, kQuantCtasPerSm) ptq_quantize_vec8_kernel
             if (b + j * S < p.B) {
                 uint2 out;
                 bool exact = !kFast;
-                if (kFast) exact = quantize8_screen(cur[j].x, cur[j].y, cur[j].z, cur[j].w, c8, out.x, out.y);
-                if (exact) quantize8_exact<kFast>(cur[j].x, cur[j].y, cur[j].z, cur[j].w, s8, rs8, d.x, d.y, out.x, out.y);
+                if (kFast) exact = quantize8_screen<kAsym>(cur[j].x, cur[j].y, cur[j].z, cur[j].w, c8, out.x, out.y, z);
+                if (exact)
+                    quantize8_exact<kFast, kAsym>(cur[j].x, cur[j].y, cur[j].z, cur[j].w, s8, rs8, d.x, d.y, out.x, out.y, z);
                 *reinterpret_cast<uint2 *>(qp + j * q_step) = out;
             }
         }
@@ -216,7 +245,7 @@ __global__ void __launch_bounds__(256, kQuantCtasPerSm) ptq_quantize_vec8_kernel
 }
 
 // Generic path: any K, any alignment; one element per thread per step.
-template <bool kFast>
+template <bool kFast, bool kAsym = false>
 __global__ void __launch_bounds__(256) ptq_quantize_scalar_kernel(QuantParams p)
 {
     const long long total = p.M * p.K;
@@ -228,11 +257,12 @@ __global__ void __launch_bounds__(256) ptq_quantize_scalar_kernel(QuantParams p)
         const __half h = p.x[i];
         const float xf = __half2float(h);
         const unsigned short bits = __half_as_ushort(h);
+        const int z = kAsym ? __ldg(p.zp + t) : 0;
         int c;
         if (kFast && (bits & 0x7c00u) != 0x7c00u)
-            c = quantize_fast(xf, __ldg(p.s + k), __ldg(p.rs + k), __ldg(p.dx + t), __ldg(p.rdx + t));
+            c = quantize_fast<kAsym>(xf, __ldg(p.s + k), __ldg(p.rs + k), __ldg(p.dx + t), __ldg(p.rdx + t), z);
         else
-            c = quantize_ieee(xf, __ldg(p.s + k), __ldg(p.dx + t));
+            c = quantize_ieee<kAsym>(xf, __ldg(p.s + k), __ldg(p.dx + t), z);
         p.q[m * p.q_pitch + k] = static_cast<int8_t>(c);
     }
 }

@@ -287,11 +287,11 @@ __device__ __forceinline__ void mma_commit_pair(uint32_t bar)
 
 // Instruction descriptor of tcgen05.mma kind::i8, dense, signed 8-bit A and B (both K-major),
 // signed 32-bit accumulator, tile M x N.  Field positions: D format [4,6) (2 = s32),
-// A format [7,10) and B format [10,13) (1 = signed 8-bit), A/B major [15],[16] (0 = K-major),
+// A format [7,10) and B format [10,13) (1 = signed 8-bit, 0 = unsigned 8-bit), A/B major [15],[16] (0 = K-major),
 // N>>3 at [17,23), M>>4 at [24,29).
-__host__ __device__ constexpr uint32_t make_idesc_s8(int M, int N)
+__host__ __device__ constexpr uint32_t make_idesc_s8(int M, int N, bool a_unsigned = false)
 {
-    return (2u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(N >> 3) << 17) |
+    return (2u << 4) | ((a_unsigned ? 0u : 1u) << 7) | (1u << 10) | (static_cast<uint32_t>(N >> 3) << 17) |
            (static_cast<uint32_t>(M >> 4) << 24);
 }
 
