@@ -264,8 +264,12 @@ def run_ours(args, specs, rank, world, local_rank):
         x_host = torch.from_numpy(wl.activations(sp, wl.ROLE_EVAL)).pin_memory()
         wq, dw, bias = wl.weights(sp)
         xcal = torch.from_numpy(wl.activations(sp, wl.ROLE_CALIB)).to(dev)
-        s, dx = ptq.calibrate(xcal, wq, dw)                      # Q0 on the GPU
-        layer = ptq.PtqLinear(wq, dw, s, dx, bias)
+        if args.scheme == "pts-asym":
+            s, dx, z = ptq.calibrate_asym(xcal, wq, dw)          # Q0 on the GPU, with zero offsets
+            layer = ptq.PtqLinear(wq, dw, s, dx, bias, act_zero=z)
+        else:
+            s, dx = ptq.calibrate(xcal, wq, dw)                  # Q0 on the GPU
+            layer = ptq.PtqLinear(wq, dw, s, dx, bias)
         x_dev = x_host.to(dev)
         y_dev = torch.empty((sp.B, sp.T, sp.N), dtype=torch.float16, device=dev)
         y_host = torch.empty((sp.B, sp.T, sp.N), dtype=torch.float16).pin_memory()
@@ -417,7 +421,7 @@ def run_ours(args, specs, rank, world, local_rank):
         "dtype": "int8", "data": "synthetic",
         "config": {"workload": args.workload, "layers": ["%s %dx%d->%d" % (sp.name, sp.M, sp.K, sp.N) for sp in specs][:8],
                    "n_layers": len(specs), "batch": sp0.B, "tokens": sp0.T, "path": args.path,
-                   "cuda_graph": bool(args.graph),
+                   "cuda_graph": bool(args.graph), "scheme": args.scheme,
                    "fused_layers": sum(1 for d in layers if d["fused"]),
                    "l2": "inputs_larger_than_l2 (%.0f MB touched per step)" % (touched / 1e6)
                    if touched > 2 * 126e6 else "working set %.0f MB fits L2: L2-warm timing" % (touched / 1e6),
@@ -455,6 +459,8 @@ def main():
     ap.add_argument("--path", default="unfused", choices=["unfused", "fused", "pair"],
                     help="unfused: quantize kernel + GEMM kernel (fastest at present, the default); "
                          "fused: PTQ_FLAG_FUSED_PROLOGUE; pair: PTQ_FLAG_CTA_PAIR")
+    ap.add_argument("--scheme", default="pts", choices=["pts", "pts-asym"],
+                    help="pts: symmetric per-token-static codes (the default); pts-asym: with a zero offset per token position")
     ap.add_argument("--graph", action="store_true",
                     help="capture one step in a CUDA graph and time replays (for launch-bound workloads such as c1)")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
