@@ -61,6 +61,8 @@ def _bind(path: str) -> ctypes.CDLL:
                                            vp, vp, vp, vp, vp, vp, vp, vp]
     L.ptqo_calibrate.restype = None
     L.ptqo_calibrate.argtypes = [vp, c_int, c_int, c_int, vp, vp, c_int, vp, vp]
+    L.ptqo_quantize_dynamic.restype = None
+    L.ptqo_quantize_dynamic.argtypes = [vp, c_long, c_int, vp, vp, vp]
     L.ptqo_quantize_asym_one.restype = ctypes.c_uint8
     L.ptqo_quantize_asym_one.argtypes = [ctypes.c_uint16, ctypes.c_float, ctypes.c_float, c_int]
     L.ptqo_quantize_asym.restype = None
@@ -294,3 +296,26 @@ def linear_forward_asym(x, T, wq, dw, s, dx, z, bias=None, rows=None, taps=False
     if rc:
         raise OverflowError("accumulator does not fit in int32")
     return (y, c, acc) if taps else y
+
+
+# --------------------------------------------------------------------------- #
+# comparator: per-token dynamic quantization                                   #
+# --------------------------------------------------------------------------- #
+def quantize_dynamic(x, s):
+    """x fp16 [M,K] -> (int8 codes [M,K], per-row steps fp32 [M]) with dx_row = max|x/s| / 127 per row."""
+    x = _c(x, np.float16)
+    M, K = x.shape
+    s = _c(s, np.float32)
+    assert s.shape == (K,)
+    q = np.empty((M, K), np.int8)
+    dx_row = np.empty(M, np.float32)
+    lib().ptqo_quantize_dynamic(_p(x), M, K, _p(s), _p(q), _p(dx_row))
+    return q, dx_row
+
+
+def linear_forward_dynamic(x, wq, dw, s, bias=None, taps=False):
+    """Dynamic comparator end to end: codes and row steps, contraction, dequantization with T = M."""
+    q, dx_row = quantize_dynamic(x, s)
+    acc = int_matmul(q, wq)
+    y = dequant(acc, q.shape[0], dx_row, dw, bias)
+    return (y, q, acc, dx_row) if taps else y

@@ -401,3 +401,39 @@ int ptqo_linear_forward_rows_asym(const uint16_t *x, long m0, long m1, int K, in
     }
     return overflow;
 }
+
+/* ========================================================================= */
+/* Comparator: per-token DYNAMIC quantization (the slower alternative the     */
+/* paper measures against PTS, Sec. 4.1 and Table "Latency comparison"): the  */
+/* step of a token row is computed from that row at run time,                 */
+/*   u[m,k] = x[m,k] / s[k],  dx_row[m] = max( max_k |u[m,k]|, 1e-5 ) / 127,  */
+/*   q[m,k] = clip( round(u[m,k] / dx_row[m]), -128, 127 ),                   */
+/* all in binary32 with the tie and special-value rules of the static case.   */
+/* The paper gives no formula for it; this is the usual symmetric min-max     */
+/* per-token rule.  The contraction and dequantization are the static ones    */
+/* with T = M and dx = dx_row.                                                */
+/* Pinned: numpy float32; every row reaches +-127 and never -128; equals the  */
+/* static quantizer fed with the row steps; power-of-two row scaling.         */
+/* ========================================================================= */
+void ptqo_quantize_dynamic(const uint16_t *x, long M, int K, const float *s, int8_t *q, float *dx_row)
+{
+    const float floor_ = 1e-5f;
+    long m;
+#pragma omp parallel for schedule(static)
+    for (m = 0; m < M; ++m) {
+        float mu = 0.0f;
+        int k;
+        for (k = 0; k < K; ++k) {
+            volatile float u = ptqo_half_to_float(x[m * K + k]) / s[k];
+            float a = fabsf(u);
+            if (a > mu) mu = a;                 /* NaN never wins the comparison */
+        }
+        if (mu < floor_) mu = floor_;
+        {
+            volatile float d = mu / 127.0f;
+            dx_row[m] = d;
+        }
+        for (k = 0; k < K; ++k)
+            q[m * K + k] = ptqo_quantize_one(x[m * K + k], s[k], dx_row[m]);
+    }
+}

@@ -69,6 +69,11 @@ MUTANTS = [
      [lambda: pins.test_calibrate_degenerate_channels_and_positions()]),
     ("calibration without the floor", "if (mu < floor_) mu = floor_;", "",
      [lambda: pins.test_calibrate_degenerate_channels_and_positions()]),
+    ("dynamic step from the raw activations", "volatile float u = ptqo_half_to_float(x[m * K + k]) / s[k];\n            float a = fabsf(u);\n            if (a > mu) mu = a;                 /* NaN never wins the comparison */",
+     "volatile float u = ptqo_half_to_float(x[m * K + k]);\n            float a = fabsf(u);\n            if (a > mu) mu = a;",
+     [lambda: pins.test_dynamic_quantizer_vs_numpy_and_invariants()]),
+    ("dynamic step over 128 levels", "volatile float d = mu / 127.0f;\n            dx_row[m] = d;", "volatile float d = mu / 128.0f;\n            dx_row[m] = d;",
+     [lambda: pins.test_dynamic_quantizer_vs_numpy_and_invariants()]),
     ("zero offset subtracted instead of added", "r = (double)nearbyintf(v) + (double)z;", "r = (double)nearbyintf(v) - (double)z;",
      [lambda: apins.test_asym_indices_ties_and_clamp()]),
     ("offset added before rounding", "r = (double)nearbyintf(v) + (double)z;", "r = (double)nearbyintf(v + (float)z);",

@@ -417,3 +417,36 @@ def test_workloads_are_deterministic_and_shaped():
     g, o = wl.structure(cfg[0][0])
     assert g[98] < 0.5 * np.median(g) and (o > 1).sum() == 4
     assert np.abs(big[:, 98]).mean() < np.abs(big).mean()
+
+
+# --------------------------------------------------------------------------- #
+# comparator: per-token dynamic quantization                                   #
+# --------------------------------------------------------------------------- #
+def test_dynamic_quantizer_vs_numpy_and_invariants():
+    spec = wl.configs()[0][0]
+    x = wl.activations(spec, wl.ROLE_EVAL, B=3).reshape(-1, spec.K)
+    x[5] = 0                                                    # a dead row: floored step, all-zero codes
+    wq, dw, _ = wl.weights(spec)
+    s, _ = oracle.calibrate(wl.activations(spec, wl.ROLE_CALIB), wq, dw)
+    q, dx_row = oracle.quantize_dynamic(x, s)
+    u = (x.astype(F32) / s[None, :]).astype(F32)
+    mu = np.maximum(np.abs(u).max(axis=1), F32(1e-5))
+    dx_np = (mu / F32(127)).astype(F32)
+    assert np.array_equal(dx_row.view(np.uint32), dx_np.view(np.uint32))
+    q_np = np.clip(np.rint((u / dx_np[:, None]).astype(F32)), -128, 127).astype(np.int8)
+    assert np.array_equal(q, q_np)
+    # every live row uses the full range and never needs the clamp
+    live = np.abs(x.astype(np.float32)).max(axis=1) > 0
+    assert np.all(np.abs(q[live].astype(np.int32)).max(axis=1) == 127) and q.min() >= -127
+    assert np.all(q[5] == 0) and dx_row[5] == F32(F32(1e-5) / F32(127))
+    # the static quantizer fed with the row steps (T = M) gives the same codes
+    assert np.array_equal(oracle.quantize(x, x.shape[0], s, dx_row), q)
+    # scaling a row by a power of two scales its step and leaves its codes alone
+    x2 = x.copy()
+    x2[7] = (x[7].astype(np.float32) * 4).astype(np.float16)
+    q2, dx2 = oracle.quantize_dynamic(x2, s)
+    assert np.array_equal(q2[7], q[7]) and dx2[7] == F32(4) * dx_row[7]
+    # end to end equals the composition with T = M
+    y, qq, acc, dd = oracle.linear_forward_dynamic(x, wq, dw, s, taps=True)
+    assert np.array_equal(acc, oracle.int_matmul(q, wq))
+    assert np.array_equal(y.view(np.uint16), oracle.dequant(acc, x.shape[0], dx_row, dw).view(np.uint16))
