@@ -156,6 +156,28 @@ ptq_status_t ptq_linear_forward(const ptq_linear_t *h, const void *x_fp16, int B
 ptq_status_t ptq_linear_forward_static(const ptq_linear_t *h, const void *x_fp16, int B, void *y_fp16,
                                        void *stream);
 
+/*
+ * Comparator: per-token DYNAMIC quantization (the alternative that Sec. 4.1 and the latency table of
+ * Sec. 6 set PTS against).  The layer's stored per-token-position steps are ignored; the step of every
+ * token row is measured on that row at run time:
+ *     u = x / s[k];   step[m] = max(max_k |u[m,k]|, 1e-5) / 127;   q = clamp(rne(u / step[m]), -128, 127)
+ *     y[m,n] = fp16(float(sum_k q[m,k] Wq[n,k]) * step[m] * dw[n] + bias[n])
+ * (binary32, same rounding and special-value rules as ptq_linear_forward).  The paper gives no
+ * formula for its dynamic baseline; this is the usual symmetric min-max rule per token.
+ *   h            a symmetric layer (ptq_linear_create); asymmetric layers give PTQ_ERR_VALUE
+ *   x_fp16, B, y_fp16, stream   as for ptq_linear_forward
+ *   workspace    device, 16-byte aligned, at least ptq_linear_workspace_bytes_dynamic(h, B) bytes
+ *                (codes, then one float per row); caller-owned, contents undefined afterwards
+ * The _debug form also copies out the codes (dense [B*T,K] int8), the int32 accumulators [B*T,N]
+ * and the row steps ([B*T] float); each tap pointer may be NULL.
+ */
+size_t ptq_linear_workspace_bytes_dynamic(const ptq_linear_t *h, int B);
+ptq_status_t ptq_linear_forward_dynamic(const ptq_linear_t *h, const void *x_fp16, int B, void *y_fp16,
+                                        void *workspace, size_t workspace_bytes, void *stream);
+ptq_status_t ptq_linear_forward_dynamic_debug(const ptq_linear_t *h, const void *x_fp16, int B, void *y_fp16,
+                                              void *q_int8_out, void *acc_int32_out, void *step_fp32_out,
+                                              void *workspace, size_t workspace_bytes, void *stream);
+
 /* 1 if PTQ_FLAG_FUSED_PROLOGUE runs the single fused kernel for this layer, 0 if it falls back. */
 int ptq_linear_fused_supported(const ptq_linear_t *h);
 

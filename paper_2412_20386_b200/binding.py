@@ -64,6 +64,12 @@ def load_library() -> ctypes.CDLL:
     L.ptq_linear_forward.argtypes = [vp, vp, ci, vp, vp, sz, cu, vp]
     L.ptq_linear_forward_static.restype = ci
     L.ptq_linear_forward_static.argtypes = [vp, vp, ci, vp, vp]
+    L.ptq_linear_workspace_bytes_dynamic.restype = sz
+    L.ptq_linear_workspace_bytes_dynamic.argtypes = [vp, ci]
+    L.ptq_linear_forward_dynamic.restype = ci
+    L.ptq_linear_forward_dynamic.argtypes = [vp, vp, ci, vp, vp, sz, vp]
+    L.ptq_linear_forward_dynamic_debug.restype = ci
+    L.ptq_linear_forward_dynamic_debug.argtypes = [vp, vp, ci, vp, vp, vp, vp, vp, sz, vp]
     L.ptq_linear_fused_supported.restype = ci
     L.ptq_linear_fused_supported.argtypes = [vp]
     L.ptq_quantize.restype = ci
@@ -206,6 +212,38 @@ class PtqLinear:
             raise ValueError("y must be a contiguous CUDA float16 tensor [B,T,N]")
         _check(self._L.ptq_linear_forward_static(self._h, x.data_ptr(), B, y.data_ptr(), _stream_ptr(stream)))
         return y
+
+    def workspace_bytes_dynamic(self, B: int) -> int:
+        return int(self._L.ptq_linear_workspace_bytes_dynamic(self._h, B))
+
+    def forward_dynamic(self, x, y=None, workspace=None, stream=None):
+        """``ptq_linear_forward_dynamic``: the per-token dynamic comparator (row steps measured at run time)."""
+        import torch
+        B = self._batch(x)
+        if y is None:
+            y = torch.empty((B, self.T, self.N), dtype=torch.float16, device=x.device)
+        if workspace is None:
+            workspace = torch.empty(self.workspace_bytes_dynamic(B), dtype=torch.uint8, device=x.device)
+        _check(self._L.ptq_linear_forward_dynamic(self._h, x.data_ptr(), B, y.data_ptr(), workspace.data_ptr(),
+                                                  workspace.numel() * workspace.element_size(),
+                                                  _stream_ptr(stream)))
+        return y
+
+    def forward_dynamic_debug(self, x, stream=None):
+        """``ptq_linear_forward_dynamic_debug``: returns (y, q int8 [B,T,K], acc int32 [B,T,N], step fp32 [B*T])."""
+        import torch
+        B = self._batch(x)
+        dev = x.device
+        y = torch.empty((B, self.T, self.N), dtype=torch.float16, device=dev)
+        q = torch.empty((B, self.T, self.K), dtype=torch.int8, device=dev)
+        acc = torch.empty((B, self.T, self.N), dtype=torch.int32, device=dev)
+        step = torch.empty(B * self.T, dtype=torch.float32, device=dev)
+        need = self.workspace_bytes_dynamic(B)
+        ws = torch.empty(need, dtype=torch.uint8, device=dev)
+        _check(self._L.ptq_linear_forward_dynamic_debug(self._h, x.data_ptr(), B, y.data_ptr(), q.data_ptr(),
+                                                        acc.data_ptr(), step.data_ptr(), ws.data_ptr(), need,
+                                                        _stream_ptr(stream)))
+        return y, q, acc, step
 
     def quantize(self, x, q=None, stream=None):
         """``ptq_quantize``: x fp16 [B,T,K] -> int8 codes [B,T,K]."""

@@ -17,7 +17,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _CSRC = os.path.join(_HERE, "csrc")
 _SO = os.path.join(_HERE, "libptq_linear.so")
 _SOURCES = ["ptq_api.cu"]
-_DEPS = ["ptq_api.cu", "ptq_gemm.cuh", "ptq_quantize.cuh", "ptq_calibrate.cuh", "ptx_sm100.cuh",
+_DEPS = ["ptq_api.cu", "ptq_gemm.cuh", "ptq_fused.cuh", "ptq_quantize.cuh", "ptq_quantize_dynamic.cuh",
+         "ptq_calibrate.cuh", "ptx_sm100.cuh",
          os.path.join("..", "..", "include", "ptq_linear.h")]
 
 

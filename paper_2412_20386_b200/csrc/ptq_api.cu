@@ -19,6 +19,7 @@
 #include "ptq_fused.cuh"
 #include "ptq_gemm.cuh"
 #include "ptq_quantize.cuh"
+#include "ptq_quantize_dynamic.cuh"
 
 namespace {
 
@@ -254,9 +255,41 @@ ptq_status_t launch_quantize(const ptq_linear *h, const void *x, long long M, vo
     return PTQ_OK;
 }
 
+// Dynamic comparator: codes to `q` and the per-row steps to `dx_row`.
+ptq_status_t launch_quantize_dynamic(const ptq_linear *h, const void *x, long long M, void *q, int q_pitch,
+                                     float *dx_row, cudaStream_t stream)
+{
+    ptq::DynQuantParams p;
+    p.x = static_cast<const __half *>(x);
+    p.q = static_cast<int8_t *>(q);
+    p.dx_row = dx_row;
+    p.s = h->d_s;
+    p.rs = h->d_rs;
+    p.M = M;
+    p.K = h->K;
+    p.q_pitch = q_pitch;
+    const bool vec = (h->K % 8 == 0) && (reinterpret_cast<uintptr_t>(x) % 16 == 0) &&
+                     (reinterpret_cast<uintptr_t>(q) % 8 == 0) && (q_pitch % 8 == 0);
+    const long long rows_per_cta = vec ? 8 * ptq::kDynRowsPerWarp : 8;
+    long long want = (M + rows_per_cta - 1) / rows_per_cta;
+    const long long cap = static_cast<long long>(h->num_sms) * 8;
+    if (want > cap) want = cap;
+    if (want < 1) want = 1;
+    if (!vec)
+        ptq::ptq_quantize_dynamic_scalar_kernel<<<static_cast<int>(want), 256, 0, stream>>>(p);
+    else if (h->fast_div)
+        ptq::ptq_quantize_dynamic_vec8_kernel<true><<<static_cast<int>(want), 256, 0, stream>>>(p);
+    else
+        ptq::ptq_quantize_dynamic_vec8_kernel<false><<<static_cast<int>(want), 256, 0, stream>>>(p);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    PTQ_CUDA(cudaGetLastError());
+    return PTQ_OK;
+}
+
 // G1+E1 launch on codes [M, Kpad] at `codes`.
+// dx_rows != nullptr: the steps are per ROW (dynamic comparator), i.e. dx = dx_rows and T = M.
 ptq_status_t launch_gemm(const ptq_linear *h, const void *codes, long long M, void *y, void *acc_out,
-                         cudaStream_t stream, bool want_pair = false)
+                         cudaStream_t stream, bool want_pair = false, const float *dx_rows = nullptr)
 {
     static std::once_flag once;
     static ptq_status_t attr_status = PTQ_OK;
@@ -285,13 +318,13 @@ ptq_status_t launch_gemm(const ptq_linear *h, const void *codes, long long M, vo
     p.M = M;
     p.N = h->N;
     p.K = h->K;
-    p.T = h->T;
+    p.T = dx_rows ? static_cast<int>(M) : h->T;
     p.BN = h->BN;
     p.n_tiles = h->n_tiles;
     p.m_tiles = static_cast<int>((M + ptq::kBM - 1) / ptq::kBM);
     p.k_blocks = h->k_blocks;
     p.last_mmas = h->last_mmas;
-    p.dx = h->d_dx;
+    p.dx = dx_rows ? dx_rows : h->d_dx;
     p.dw = h->d_dw;
     p.bias = h->d_bias;
     p.y = static_cast<__half *>(y);
@@ -791,6 +824,55 @@ ptq_status_t ptq_linear_forward_static(const ptq_linear_t *h, const void *x_fp16
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if ((st = launch_quantize(h, x_fp16, M, scratch, h->Kpad, s)) != PTQ_OK) return st;
     return launch_gemm_any(h, scratch, M, y_fp16, nullptr, s);
+}
+
+static size_t dynamic_codes_bytes(const ptq_linear *h, long long M)
+{
+    return (static_cast<size_t>(M) * h->Kpad + 255) / 256 * 256;
+}
+
+size_t ptq_linear_workspace_bytes_dynamic(const ptq_linear_t *h, int B)
+{
+    if (!h || B < 1) return 0;
+    const long long M = static_cast<long long>(B) * h->T;
+    return dynamic_codes_bytes(h, M) + static_cast<size_t>(M) * sizeof(float);
+}
+
+ptq_status_t ptq_linear_forward_dynamic_debug(const ptq_linear_t *h, const void *x_fp16, int B, void *y_fp16,
+                                              void *q_int8_out, void *acc_int32_out, void *step_fp32_out,
+                                              void *workspace, size_t workspace_bytes, void *stream)
+{
+    ptq_status_t st = validate_forward(h, x_fp16, B, y_fp16);
+    if (st != PTQ_OK) return st;
+    if (h->asym) return fail(PTQ_ERR_VALUE, "the dynamic comparator is defined for symmetric layers only");
+    const long long M = static_cast<long long>(B) * h->T;
+    const size_t codes = dynamic_codes_bytes(h, M);
+    const size_t need = codes + static_cast<size_t>(M) * sizeof(float);
+    if (!workspace) return fail(PTQ_ERR_NULL, "workspace must not be NULL");
+    if (workspace_bytes < need)
+        return fail(PTQ_ERR_SHAPE, "workspace has %zu bytes, %zu needed", workspace_bytes, need);
+    if (reinterpret_cast<uintptr_t>(workspace) % 16) return fail(PTQ_ERR_ALIGN, "workspace must be 16-byte aligned");
+    if (ranges_overlap(workspace, need, y_fp16, static_cast<size_t>(M) * h->N * 2) ||
+        ranges_overlap(workspace, need, x_fp16, static_cast<size_t>(M) * h->K * 2))
+        return fail(PTQ_ERR_VALUE, "workspace overlaps x or y");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    float *dx_row = reinterpret_cast<float *>(static_cast<unsigned char *>(workspace) + codes);
+    if ((st = launch_quantize_dynamic(h, x_fp16, M, workspace, h->Kpad, dx_row, s)) != PTQ_OK) return st;
+    if ((st = launch_gemm(h, workspace, M, y_fp16, acc_int32_out, s, false, dx_row)) != PTQ_OK) return st;
+    if (q_int8_out)
+        PTQ_CUDA(cudaMemcpy2DAsync(q_int8_out, h->K, workspace, h->Kpad, h->K, static_cast<size_t>(M),
+                                   cudaMemcpyDeviceToDevice, s));
+    if (step_fp32_out)
+        PTQ_CUDA(cudaMemcpyAsync(step_fp32_out, dx_row, static_cast<size_t>(M) * sizeof(float),
+                                 cudaMemcpyDeviceToDevice, s));
+    return PTQ_OK;
+}
+
+ptq_status_t ptq_linear_forward_dynamic(const ptq_linear_t *h, const void *x_fp16, int B, void *y_fp16,
+                                        void *workspace, size_t workspace_bytes, void *stream)
+{
+    return ptq_linear_forward_dynamic_debug(h, x_fp16, B, y_fp16, nullptr, nullptr, nullptr, workspace,
+                                            workspace_bytes, stream);
 }
 
 ptq_status_t ptq_linear_device_status(const ptq_linear_t *h)
