@@ -273,21 +273,27 @@ def run_ours(args, specs, rank, world, local_rank):
         x_dev = x_host.to(dev)
         y_dev = torch.empty((sp.B, sp.T, sp.N), dtype=torch.float16, device=dev)
         y_host = torch.empty((sp.B, sp.T, sp.N), dtype=torch.float16).pin_memory()
-        ws_bytes = layer.workspace_bytes(sp.B, flags)
+        ws_bytes = layer.workspace_bytes_dynamic(sp.B) if args.scheme == "dynamic" else layer.workspace_bytes(sp.B, flags)
         ws = torch.empty(max(ws_bytes, 16), dtype=torch.uint8, device=dev)
         layers.append(dict(spec=sp, layer=layer, x_host=x_host, x=x_dev, y=y_dev, y_host=y_host, ws=ws,
                            fused=bool((flags & ptq.FLAG_FUSED_PROLOGUE) and layer.fused_supported())))
     step_ops = sum(layer_ops(d["spec"], d["spec"].B) for d in layers)
     touched = sum(d["x"].numel() * 2 + d["y"].numel() * 2 for d in layers)
 
+    def forward(d):
+        if args.scheme == "dynamic":
+            d["layer"].forward_dynamic(d["x"], y=d["y"], workspace=d["ws"])
+        else:
+            d["layer"].forward(d["x"], y=d["y"], workspace=d["ws"], flags=flags)
+
     def step():
         for d in layers:
-            d["layer"].forward(d["x"], y=d["y"], workspace=d["ws"], flags=flags)
+            forward(d)
 
     def step_e2e():
         for d in layers:
             d["x"].copy_(d["x_host"], non_blocking=True)
-            d["layer"].forward(d["x"], y=d["y"], workspace=d["ws"], flags=flags)
+            forward(d)
             d["y_host"].copy_(d["y"], non_blocking=True)
 
     def barrier():
@@ -367,6 +373,17 @@ def run_ours(args, specs, rank, world, local_rank):
             avg, mn, med = event_times_ms(torch, lambda: layer.forward(d["x"], y=d["y"], workspace=d["ws"], flags=flags), iters)
             byts = 2.0 * M * K + N * K + 2.0 * M * N
             kernels.append(dict(kernel="ptq_fused_linear_kernel", layer=tag, ms=avg, ms_min=mn, ops=2.0 * M * K * N, bytes=byts))
+        elif args.scheme == "dynamic":
+            # the row-step quantizer has no entry point of its own: forward minus the GEMM timed alone
+            pitch = layer.code_pitch()
+            forward(d)
+            tot, _, _ = event_times_ms(torch, lambda: forward(d), iters)
+            g_avg, g_mn, _ = event_times_ms(torch, lambda: layer.gemm_dequant(d["ws"][:M * pitch], sp.B, y=d["y"]), iters)
+            q_ms = max(tot - g_avg, 1e-6)
+            kernels.append(dict(kernel="ptq_quantize_dynamic_kernel", layer=tag, ms=q_ms, ms_min=q_ms, ops=0.0,
+                                bytes=3.0 * M * K + 4.0 * M))
+            kernels.append(dict(kernel="ptq_gemm_dequant_kernel", layer=tag, ms=g_avg, ms_min=g_mn, ops=2.0 * M * K * N,
+                                bytes=1.0 * M * K + N * K + 2.0 * M * N))
         else:
             pitch = layer.code_pitch()
             codes = d["ws"][:M * pitch]
@@ -404,7 +421,8 @@ def run_ours(args, specs, rank, world, local_rank):
     roof.update({"kernel": dom["kernel"], "layer": dom["layer"], "ms_per_launch": dom["ms"],
                  "peak_source": "%s (%s)" % (("2 x bf16_tflops_sustained" if dom["bound"] == "tensor" else "hbm_gbs"),
                                              peaks_kind),
-                 "traffic": TRAFFIC.get((dom["kernel"], args.workload, dom["layer"].split(".")[-1]))})
+                 "traffic": TRAFFIC.get((dom["kernel"], args.workload, dom["layer"].split(".")[-1]))
+                 if args.scheme == "pts" else None})
 
     # ---- CPU oracle baseline on a bounded sample -------------------------------------------
     import oracle
@@ -442,10 +460,10 @@ def run_ours(args, specs, rank, world, local_rank):
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised
 # under profiles/; keyed by (kernel, workload, layer).  An entry is removed when its kernel changes.
 TRAFFIC = {
-    ("ptq_gemm_dequant_kernel", "c3", "in_proj"): 41.241088e6 + 255.717632e6,
-    ("ptq_gemm_dequant_kernel", "c3", "out_proj"): 78.695936e6 + 34.413312e6,
-    ("ptq_quantize_kernel", "c3", "in_proj"): 77.491456e6 + 7.729664e6,
-    ("ptq_quantize_kernel", "c3", "out_proj"): 154.964736e6 + 24.675072e6,
+    ("ptq_gemm_dequant_kernel", "c3", "in_proj"): 41.175296e6 + 255.838976e6,
+    ("ptq_gemm_dequant_kernel", "c3", "out_proj"): 78.698240e6 + 34.846976e6,
+    ("ptq_quantize_kernel", "c3", "in_proj"): 77.490688e6 + 6.991104e6,
+    ("ptq_quantize_kernel", "c3", "out_proj"): 154.978560e6 + 24.388096e6,
 }
 
 
@@ -459,8 +477,9 @@ def main():
     ap.add_argument("--path", default="unfused", choices=["unfused", "fused", "pair"],
                     help="unfused: quantize kernel + GEMM kernel (fastest at present, the default); "
                          "fused: PTQ_FLAG_FUSED_PROLOGUE; pair: PTQ_FLAG_CTA_PAIR")
-    ap.add_argument("--scheme", default="pts", choices=["pts", "pts-asym"],
-                    help="pts: symmetric per-token-static codes (the default); pts-asym: with a zero offset per token position")
+    ap.add_argument("--scheme", default="pts", choices=["pts", "pts-asym", "dynamic"],
+                    help="pts: symmetric per-token-static codes (the default); pts-asym: with a zero offset per token "
+                         "position; dynamic: the per-token dynamic comparator (row steps measured at run time)")
     ap.add_argument("--graph", action="store_true",
                     help="capture one step in a CUDA graph and time replays (for launch-bound workloads such as c1)")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)

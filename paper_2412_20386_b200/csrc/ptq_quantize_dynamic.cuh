@@ -31,7 +31,13 @@ struct DynQuantParams {
     int q_pitch;
 };
 
-constexpr int kDynRowsPerWarp = 4;
+#ifndef PTQ_DYN_ROWS_PER_WARP
+#define PTQ_DYN_ROWS_PER_WARP 2
+#endif
+#ifndef PTQ_DYN_CTAS_PER_SM
+#define PTQ_DYN_CTAS_PER_SM 4
+#endif
+constexpr int kDynRowsPerWarp = PTQ_DYN_ROWS_PER_WARP;
 constexpr float kDynScaleLo = 9.313225746154785e-10f;   // 2^-30
 constexpr float kDynScaleHi = 1073741824.0f;            // 2^30
 
@@ -65,7 +71,7 @@ __device__ __forceinline__ float chunk_absmax(const uint4 &v, const float4 &s0, 
 // A warp takes kDynRowsPerWarp consecutive rows at a time so that one load of s / RN(1/s) serves
 // several rows; lanes take consecutive 8-channel chunks (512-byte loads, 256-byte stores per warp).
 template <bool kFast>
-__global__ void __launch_bounds__(256) ptq_quantize_dynamic_vec8_kernel(DynQuantParams p)
+__global__ void __launch_bounds__(256, PTQ_DYN_CTAS_PER_SM) ptq_quantize_dynamic_vec8_kernel(DynQuantParams p)
 {
     constexpr int R = kDynRowsPerWarp;
     const int lane = threadIdx.x & 31;
