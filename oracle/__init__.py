@@ -61,6 +61,8 @@ def _bind(path: str) -> ctypes.CDLL:
                                            vp, vp, vp, vp, vp, vp, vp, vp]
     L.ptqo_calibrate.restype = None
     L.ptqo_calibrate.argtypes = [vp, c_int, c_int, c_int, vp, vp, c_int, vp, vp]
+    L.ptqo_search_act_step.restype = None
+    L.ptqo_search_act_step.argtypes = [vp, c_int, c_int, c_int, vp, vp, c_int, c_int, vp, vp, vp]
     L.ptqo_quantize_dynamic.restype = None
     L.ptqo_quantize_dynamic.argtypes = [vp, c_long, c_int, vp, vp, vp]
     L.ptqo_quantize_asym_one.restype = ctypes.c_uint8
@@ -319,3 +321,22 @@ def linear_forward_dynamic(x, wq, dw, s, bias=None, taps=False):
     acc = int_matmul(q, wq)
     y = dequant(acc, q.shape[0], dx_row, dw, bias)
     return (y, q, acc, dx_row) if taps else y
+
+
+# --------------------------------------------------------------------------- #
+# step-size search (Sec. 5.2, second stage)                                    #
+# --------------------------------------------------------------------------- #
+def search_act_step(xcal, s, base, n_grid=100, j_lo=20):
+    """xcal fp16 [Bc,T,K] -> (dx fp32 [T], best int32 [T], loss fp64 [T, n_grid-j_lo+1]):
+    per token position the candidate base[t]*j/n_grid (j_lo <= j <= n_grid) of least squared error."""
+    xcal = _c(xcal, np.float16)
+    Bc, T, K = xcal.shape
+    s = _c(s, np.float32)
+    base = _c(base, np.float32)
+    assert s.shape == (K,) and base.shape == (T,) and 1 <= j_lo <= n_grid
+    C = n_grid - j_lo + 1
+    loss = np.empty((T, C), np.float64)
+    best = np.empty(T, np.int32)
+    dx = np.empty(T, np.float32)
+    lib().ptqo_search_act_step(_p(xcal), Bc, T, K, _p(s), _p(base), n_grid, j_lo, _p(loss), _p(best), _p(dx))
+    return dx, best, loss

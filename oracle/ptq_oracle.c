@@ -437,3 +437,62 @@ void ptqo_quantize_dynamic(const uint16_t *x, long M, int K, const float *s, int
             q[m * K + k] = ptqo_quantize_one(x[m * K + k], s[k], dx_row[m]);
     }
 }
+
+/* ========================================================================= */
+/* Step-size search (Sec. 5.2, second stage; the "+Truncation" row of the     */
+/* ablation table): per token position, the step that minimises the L2        */
+/* distance between the smoothed calibration activations and their            */
+/* dequantized codes, searched over a grid of truncation ratios.  The paper   */
+/* states the loss and that it is a grid search, not the grid; here           */
+/*   Delta[t,j] = base[t] * (j / n_grid)        j = j_lo .. n_grid            */
+/*   u = x / s[k],  q = clip(round(u / Delta[t,j]), -128, 127)                */
+/*   e = u - Delta[t,j] * q     (one rounding: fused multiply-add, binary32)  */
+/*   loss[t,j] = sum_{b,k} e^2  (binary64 sum; non-finite u are skipped)      */
+/*   best[t] = the j of least loss, the LARGEST such j on equal losses        */
+/* with base[t] normally the min-max step (j = n_grid is "no truncation").    */
+/* Pinned: exact rational brute force on tiny inputs; zero loss on grid       */
+/* points; Delta^2/12 law without clipping; truncation wins with an outlier.  */
+/* ========================================================================= */
+void ptqo_search_act_step(const uint16_t *xcal, int Bc, int T, int K, const float *s, const float *base,
+                          int n_grid, int j_lo, double *loss, int32_t *best, float *dx)
+{
+    const int C = n_grid - j_lo + 1;
+    int t;
+#pragma omp parallel for schedule(static)
+    for (t = 0; t < T; ++t) {
+        int j, best_j = n_grid;
+        double best_loss = 0.0;
+        for (j = n_grid; j >= j_lo; --j) {
+            volatile float ratio = (float)j / (float)n_grid;
+            volatile float delta = base[t] * ratio;
+            double acc = 0.0;
+            int b, k;
+            for (b = 0; b < Bc; ++b) {
+                long m = (long)b * T + t;
+                for (k = 0; k < K; ++k) {
+                    volatile float u = ptqo_half_to_float(xcal[m * K + k]) / s[k];
+                    volatile float v;
+                    float r, e;
+                    if (!isfinite(u)) continue;
+                    v = u / delta;
+                    r = nearbyintf(v);
+                    if (r > 127.0f) r = 127.0f;
+                    if (r < -128.0f) r = -128.0f;
+                    e = fmaf(-delta, r, u);
+                    acc += (double)e * (double)e;
+                }
+            }
+            loss[(long)t * C + (j - j_lo)] = acc;
+            if (j == n_grid || acc < best_loss) {     /* descending j and strict '<': ties keep the larger j */
+                best_loss = acc;
+                best_j = j;
+            }
+        }
+        best[t] = best_j;
+        {
+            volatile float ratio = (float)best_j / (float)n_grid;
+            volatile float delta = base[t] * ratio;
+            dx[t] = delta;
+        }
+    }
+}

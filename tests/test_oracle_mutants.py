@@ -8,6 +8,7 @@ import pytest
 import oracle
 import test_oracle_asym_pins as apins
 import test_oracle_pins as pins
+import test_oracle_search_pins as spins
 
 SRC = open(os.path.join(os.path.dirname(oracle.__file__), "ptq_oracle.c")).read()
 
@@ -69,6 +70,26 @@ MUTANTS = [
      [lambda: pins.test_calibrate_degenerate_channels_and_positions()]),
     ("calibration without the floor", "if (mu < floor_) mu = floor_;", "",
      [lambda: pins.test_calibrate_degenerate_channels_and_positions()]),
+    ("search: error with the wrong sign of the dequantized value", "e = fmaf(-delta, r, u);", "e = fmaf(delta, r, u);",
+     [lambda: spins.test_search_zero_loss_on_grid_points_and_ties_keep_the_largest_ratio()]),
+    ("search: L1 instead of L2 loss", "acc += (double)e * (double)e;", "acc += fabs((double)e);",
+     [lambda: spins.test_search_loss_follows_the_uniform_rounding_error_law()]),
+    ("search: codes not clipped", "if (r < -128.0f) r = -128.0f;\n                    e = fmaf", "e = fmaf",
+     [lambda: spins.test_search_truncates_when_an_outlier_stretches_the_range()]),
+    ("search: ties go to the smallest ratio", "if (j == n_grid || acc < best_loss) {", "if (j == n_grid || acc <= best_loss) {",
+     [lambda: spins.test_search_zero_loss_on_grid_points_and_ties_keep_the_largest_ratio()]),
+    ("search: candidate grid shifted by one", "volatile float ratio = (float)j / (float)n_grid;\n            volatile float delta = base[t] * ratio;\n            double acc",
+     "volatile float ratio = (float)(j - 1) / (float)n_grid;\n            volatile float delta = base[t] * ratio;\n            double acc",
+     [lambda: spins.test_search_matches_exact_rational_brute_force()]),
+    ("search: non-finite activations poison the loss", "if (!isfinite(u)) continue;", "",
+     [lambda: spins.test_search_skips_non_finite_values_and_uses_the_pinned_quantizer()]),
+    ("search: largest loss chosen", "if (j == n_grid || acc < best_loss) {", "if (j == n_grid || acc > best_loss) {",
+     [lambda: spins.test_search_truncates_when_an_outlier_stretches_the_range()]),
+    ("search: smoothing scale ignored", "volatile float u = ptqo_half_to_float(xcal[m * K + k]) / s[k];\n                    volatile float v;",
+     "volatile float u = ptqo_half_to_float(xcal[m * K + k]);\n                    volatile float v;",
+     [lambda: spins.test_search_matches_exact_rational_brute_force()]),
+    ("search: returned step is the full step", "volatile float ratio = (float)best_j / (float)n_grid;", "volatile float ratio = 1.0f;",
+     [lambda: spins.test_search_truncates_when_an_outlier_stretches_the_range()]),
     ("dynamic step from the raw activations", "volatile float u = ptqo_half_to_float(x[m * K + k]) / s[k];\n            float a = fabsf(u);\n            if (a > mu) mu = a;                 /* NaN never wins the comparison */",
      "volatile float u = ptqo_half_to_float(x[m * K + k]);\n            float a = fabsf(u);\n            if (a > mu) mu = a;",
      [lambda: pins.test_dynamic_quantizer_vs_numpy_and_invariants()]),
