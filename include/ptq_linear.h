@@ -231,6 +231,33 @@ ptq_status_t ptq_calibrate(int K, int N, int T, const void *xcal_fp16, int Bc,
                            float *smooth_out, float *act_step_out, void *stream);
 
 /*
+ * Step-size search (Sec. 5.2, second stage; the "+Truncation" row of the ablation): for every token
+ * position the candidate step
+ *     Delta[t,j] = base_step[t] * (j / n_grid),   j = j_lo .. n_grid
+ * that minimises the squared distance between the smoothed calibration activations u = x / s[k] and
+ * their dequantized codes,
+ *     loss[t,j] = sum_{b,k} (u - Delta[t,j] * clip(rne(u / Delta[t,j]), -128, 127))^2 ,
+ * the largest j on equal losses.  Steps, quotients and the element error are binary32 (the error with
+ * one rounding, as a fused multiply-add); the sum is binary64 and its order is fixed for a given
+ * shape, but it is not the sequential order, so two candidates whose losses agree to about 1e-13
+ * relative may be ranked either way.  Non-finite u do not enter the loss.  The paper states the
+ * objective and that it is a grid search; the grid is this library's choice (a common one is
+ * n_grid = 100, j_lo = 20 with base_step the min-max steps of ptq_calibrate: j = n_grid is "no
+ * truncation").
+ *   xcal_fp16     device, [Bc,T,K] contiguous binary16
+ *   smooth        host, [K], positive finite;  base_step  host, [T], in [1e-30, inf)
+ *   n_grid, j_lo  1 <= j_lo <= n_grid <= PTQ_MAX_SEARCH_GRID
+ *   act_step_out  host, [T]: the chosen steps
+ *   best_out      host, [T] int32: the chosen j, or NULL
+ *   loss_out      host, [T, n_grid - j_lo + 1] binary64: every loss, or NULL
+ * Allocates temporary device memory and synchronises the stream before returning.
+ */
+#define PTQ_MAX_SEARCH_GRID 4096
+ptq_status_t ptq_search_act_step(int K, int T, const void *xcal_fp16, int Bc, const float *smooth,
+                                 const float *base_step, int n_grid, int j_lo, float *act_step_out,
+                                 int32_t *best_out, double *loss_out, void *stream);
+
+/*
  * Q0 for asymmetric layers: s[k] as in ptq_calibrate; per token position the range [lo, hi] of x/s over
  * the calibration batch, widened to contain zero; dx[t] = max(hi - lo, 1e-5) / 255 and
  * z[t] = clip(rne(-lo / dx[t]), 0, 255)  (Delta_X and eps_X of Sec. 2.3 per token position, Sec. 5.1).

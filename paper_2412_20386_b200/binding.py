@@ -82,6 +82,8 @@ def load_library() -> ctypes.CDLL:
     L.ptq_linear_forward_debug.argtypes = [vp, vp, ci, vp, vp, vp, vp, sz, cu, vp]
     L.ptq_calibrate.restype = ci
     L.ptq_calibrate.argtypes = [ci, ci, ci, vp, ci, vp, vp, vp, vp, vp]
+    L.ptq_search_act_step.restype = ci
+    L.ptq_search_act_step.argtypes = [ci, ci, vp, ci, vp, vp, ci, ci, vp, vp, vp, vp]
     L.ptq_linear_describe.restype = ci
     L.ptq_linear_describe.argtypes = [vp, ctypes.c_char_p, ci]
     L.ptq_linear_device_status.restype = ci
@@ -325,3 +327,21 @@ def calibrate_asym(xcal, w_q, w_step, stream=None):
     _check(L.ptq_calibrate_asym(K, N, T, xcal.data_ptr(), Bc, _hp(w_q), _hp(w_step), _hp(s), _hp(dx), _hp(z),
                                 _stream_ptr(stream)))
     return s, dx, z
+
+
+def search_act_step(xcal, smooth, base_step, n_grid: int = 100, j_lo: int = 20, want_loss: bool = False, stream=None):
+    """``ptq_search_act_step``: device fp16 [Bc,T,K] -> (dx fp32 [T], best j int32 [T], loss fp64 [T,C] or None)."""
+    import torch
+    L = load_library()
+    if xcal.dtype != torch.float16 or not xcal.is_cuda or not xcal.is_contiguous() or xcal.dim() != 3:
+        raise ValueError("xcal must be a contiguous CUDA float16 tensor [Bc,T,K]")
+    Bc, T, K = (int(v) for v in xcal.shape)
+    smooth = _host(smooth, np.float32, (K,))
+    base_step = _host(base_step, np.float32, (T,))
+    dx = np.empty(T, np.float32)
+    best = np.empty(T, np.int32)
+    loss = np.empty((T, max(n_grid - j_lo + 1, 1)), np.float64) if want_loss else None
+    _check(L.ptq_search_act_step(K, T, xcal.data_ptr(), Bc, smooth.ctypes.data, base_step.ctypes.data, n_grid, j_lo,
+                                 dx.ctypes.data, best.ctypes.data,
+                                 loss.ctypes.data if loss is not None else None, _stream_ptr(stream)))
+    return dx, best, loss

@@ -826,6 +826,65 @@ ptq_status_t ptq_linear_forward_static(const ptq_linear_t *h, const void *x_fp16
     return launch_gemm_any(h, scratch, M, y_fp16, nullptr, s);
 }
 
+ptq_status_t ptq_search_act_step(int K, int T, const void *xcal_fp16, int Bc, const float *smooth,
+                                 const float *base_step, int n_grid, int j_lo, float *act_step_out,
+                                 int32_t *best_out, double *loss_out, void *stream)
+{
+    if (!xcal_fp16 || !smooth || !base_step || !act_step_out)
+        return fail(PTQ_ERR_NULL, "search: pointers must not be NULL");
+    if (K < 1 || K > PTQ_MAX_K || T < 1 || T > PTQ_MAX_T || Bc < 1 ||
+        static_cast<long long>(Bc) * K > 0x7fffffffll)
+        return fail(PTQ_ERR_SHAPE, "search: dimensions out of range (K=%d T=%d Bc=%d)", K, T, Bc);
+    if (n_grid < 1 || n_grid > PTQ_MAX_SEARCH_GRID || j_lo < 1 || j_lo > n_grid)
+        return fail(PTQ_ERR_VALUE, "search: need 1 <= j_lo <= n_grid <= %d (got j_lo=%d n_grid=%d)",
+                    PTQ_MAX_SEARCH_GRID, j_lo, n_grid);
+    if (reinterpret_cast<uintptr_t>(xcal_fp16) % 2) return fail(PTQ_ERR_ALIGN, "xcal must be 2-byte aligned");
+    for (int k = 0; k < K; ++k)
+        if (!(smooth[k] > 0.0f) || !std::isfinite(smooth[k]))
+            return fail(PTQ_ERR_VALUE, "search: smooth[%d] = %g is not positive and finite", k, smooth[k]);
+    for (int t = 0; t < T; ++t)
+        if (!(base_step[t] >= 1e-30f) || !std::isfinite(base_step[t]))
+            return fail(PTQ_ERR_VALUE, "search: base_step[%d] = %g is not in [1e-30, inf)", t, base_step[t]);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int C = n_grid - j_lo + 1;
+    float *d_f = nullptr;      // [K] s, [T] base, [T] dx
+    int *d_best = nullptr;     // [T]
+    double *d_loss = nullptr;  // [T, C]
+    auto body = [&]() -> ptq_status_t {
+        PTQ_CUDA(cudaMalloc(reinterpret_cast<void **>(&d_f), sizeof(float) * (K + 2 * static_cast<size_t>(T))));
+        PTQ_CUDA(cudaMalloc(reinterpret_cast<void **>(&d_best), sizeof(int) * static_cast<size_t>(T)));
+        PTQ_CUDA(cudaMalloc(reinterpret_cast<void **>(&d_loss), sizeof(double) * static_cast<size_t>(T) * C));
+        PTQ_CUDA(cudaMemcpyAsync(d_f, smooth, sizeof(float) * K, cudaMemcpyHostToDevice, s));
+        PTQ_CUDA(cudaMemcpyAsync(d_f + K, base_step, sizeof(float) * T, cudaMemcpyHostToDevice, s));
+        ptq::SearchParams p;
+        p.x = static_cast<const __half *>(xcal_fp16);
+        p.s = d_f;
+        p.base = d_f + K;
+        p.loss = d_loss;
+        p.Bc = Bc;
+        p.T = T;
+        p.K = K;
+        p.n_grid = n_grid;
+        p.j_lo = j_lo;
+        const dim3 grid(static_cast<unsigned>(T), static_cast<unsigned>((C + ptq::kSearchCandPerBlock - 1) / ptq::kSearchCandPerBlock));
+        ptq::ptq_search_loss_kernel<<<grid, ptq::kSearchThreads, 0, s>>>(p);
+        ptq::ptq_search_pick_kernel<<<(T + 127) / 128, 128, 0, s>>>(d_loss, d_f + K, T, n_grid, j_lo, d_best, d_f + K + T);
+        g_launches.fetch_add(2, std::memory_order_relaxed);
+        PTQ_CUDA(cudaGetLastError());
+        PTQ_CUDA(cudaMemcpyAsync(act_step_out, d_f + K + T, sizeof(float) * T, cudaMemcpyDeviceToHost, s));
+        if (best_out) PTQ_CUDA(cudaMemcpyAsync(best_out, d_best, sizeof(int) * T, cudaMemcpyDeviceToHost, s));
+        if (loss_out)
+            PTQ_CUDA(cudaMemcpyAsync(loss_out, d_loss, sizeof(double) * static_cast<size_t>(T) * C, cudaMemcpyDeviceToHost, s));
+        PTQ_CUDA(cudaStreamSynchronize(s));
+        return PTQ_OK;
+    };
+    const ptq_status_t st = body();
+    cudaFree(d_f);
+    cudaFree(d_best);
+    cudaFree(d_loss);
+    return st;
+}
+
 static size_t dynamic_codes_bytes(const ptq_linear *h, long long M)
 {
     return (static_cast<size_t>(M) * h->Kpad + 255) / 256 * 256;

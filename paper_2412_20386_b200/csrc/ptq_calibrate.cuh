@@ -138,4 +138,91 @@ __global__ void __launch_bounds__(128) ptq_calib_step_asym_kernel(const unsigned
     z[t] = static_cast<int>(fminf(fmaxf(zr, 0.0f), 255.0f));
 }
 
+// --- step-size search (Sec. 5.2, second stage; "+Truncation" in the ablation) ----------------------
+// Per token position t and candidate j (j_lo <= j <= n_grid):
+//   Delta = RN(base[t] * RN(j / n_grid)),  u = RN(x / s[k]),  q = clip(rne(RN(u / Delta)), -128, 127)
+//   e = RN(u - Delta * q)  (one fused multiply-add),  loss[t,j] = sum_{b,k} e^2 in binary64,
+// non-finite u skipped.  One block per (position, group of kSearchCandPerBlock candidates); threads
+// stride over the Bc*K elements of the position, keep one binary64 partial sum per candidate, and the
+// block reduces them in a fixed order (shuffles, then warp by warp), so a launch is reproducible.
+constexpr int kSearchCandPerBlock = 8;
+constexpr int kSearchThreads = 256;
+
+struct SearchParams {
+    const __half *x;     // [Bc,T,K]
+    const float *s;      // [K]
+    const float *base;   // [T]
+    double *loss;        // [T, n_grid - j_lo + 1]
+    int Bc, T, K;
+    int n_grid, j_lo;
+};
+
+__device__ __forceinline__ float search_candidate_step(float base, int j, int n_grid)
+{
+    return __fmul_rn(base, __fdiv_rn(static_cast<float>(j), static_cast<float>(n_grid)));
+}
+
+__global__ void __launch_bounds__(kSearchThreads) ptq_search_loss_kernel(SearchParams p)
+{
+    constexpr int C = kSearchCandPerBlock;
+    __shared__ double partial[kSearchThreads / 32][C];
+    const int t = blockIdx.x;
+    const int j0 = p.j_lo + static_cast<int>(blockIdx.y) * C;
+    const int ncand = min(C, p.n_grid - j0 + 1);
+    const float base = __ldg(p.base + t);
+    float delta[C];
+    double acc[C];
+#pragma unroll
+    for (int c = 0; c < C; ++c) {
+        delta[c] = search_candidate_step(base, min(j0 + c, p.n_grid), p.n_grid);
+        acc[c] = 0.0;
+    }
+    const int per_pos = p.Bc * p.K;
+    for (int i = threadIdx.x; i < per_pos; i += kSearchThreads) {
+        const int b = i / p.K;
+        const int k = i - b * p.K;
+        const float xf = __half2float(p.x[(static_cast<long long>(b) * p.T + t) * p.K + k]);
+        const float u = __fdiv_rn(xf, __ldg(p.s + k));
+        if (!(fabsf(u) <= 3.402823466e38f)) continue;          // inf and NaN do not enter the loss
+#pragma unroll
+        for (int c = 0; c < C; ++c) {
+            float r = rintf(__fdiv_rn(u, delta[c]));
+            r = fminf(fmaxf(r, -128.0f), 127.0f);
+            const double e = static_cast<double>(__fmaf_rn(-delta[c], r, u));
+            acc[c] = fma(e, e, acc[c]);
+        }
+    }
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int c = 0; c < C; ++c) {
+        double v = acc[c];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        if (lane == 0) partial[warp][c] = v;
+    }
+    __syncthreads();
+    if (threadIdx.x < ncand) {
+        double v = 0.0;
+        for (int w = 0; w < kSearchThreads / 32; ++w) v += partial[w][threadIdx.x];
+        p.loss[static_cast<long long>(t) * (p.n_grid - p.j_lo + 1) + (j0 - p.j_lo) + threadIdx.x] = v;
+    }
+}
+
+// The candidate of least loss per position, the largest j among equals (scan from n_grid down, strict <).
+__global__ void __launch_bounds__(128) ptq_search_pick_kernel(const double *loss, const float *base, int T, int n_grid,
+                                                              int j_lo, int *best, float *dx)
+{
+    const int t = blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= T) return;
+    const double *row = loss + static_cast<long long>(t) * (n_grid - j_lo + 1);
+    int bj = n_grid;
+    double bl = row[n_grid - j_lo];
+    for (int j = n_grid - 1; j >= j_lo; --j) {
+        const double l = row[j - j_lo];
+        if (l < bl) { bl = l; bj = j; }
+    }
+    best[t] = bj;
+    dx[t] = search_candidate_step(__ldg(base + t), bj, n_grid);
+}
+
 }  // namespace ptq
