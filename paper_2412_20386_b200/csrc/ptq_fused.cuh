@@ -279,25 +279,18 @@ ptq_fused_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                     const long long m = m0 + 16 * j;
                     uint4 out = make_uint4(0, 0, 0, 0);      // rows beyond M and channels beyond K hold zero codes
                     if (col_ok && m < p.M) {
-                        float c8[8];
-                        bool exact = !kFast;
+                        float c8[8] = {};
                         if (kFast) {
 #pragma unroll
                             for (int i = 0; i < 8; ++i) c8[i] = __fmul_rn(rs16[i], dj[j].y);
-                            exact = quantize8_screen(u[j][0].x, u[j][0].y, u[j][0].z, u[j][0].w, c8, out.x, out.y);
                         }
-                        if (exact)
-                            quantize8_exact<kFast>(u[j][0].x, u[j][0].y, u[j][0].z, u[j][0].w, fp.s + kcol, fp.rs + kcol,
-                                                   dj[j].x, dj[j].y, out.x, out.y);
-                        exact = !kFast;
+                        const uint2 o0 = quantize8<kFast, false>(u[j][0], c8, fp.s + kcol, fp.rs + kcol, dj[j].x, dj[j].y, 0);
                         if (kFast) {
 #pragma unroll
                             for (int i = 0; i < 8; ++i) c8[i] = __fmul_rn(rs16[8 + i], dj[j].y);
-                            exact = quantize8_screen(u[j][1].x, u[j][1].y, u[j][1].z, u[j][1].w, c8, out.z, out.w);
                         }
-                        if (exact)
-                            quantize8_exact<kFast>(u[j][1].x, u[j][1].y, u[j][1].z, u[j][1].w, fp.s + kcol + 8,
-                                                   fp.rs + kcol + 8, dj[j].x, dj[j].y, out.z, out.w);
+                        const uint2 o1 = quantize8<kFast, false>(u[j][1], c8, fp.s + kcol + 8, fp.rs + kcol + 8, dj[j].x, dj[j].y, 0);
+                        out = make_uint4(o0.x, o0.y, o1.x, o1.y);
                     }
                     // 128-byte swizzle of the K-major operand layout: 16-byte chunk index XOR (row mod 8)
                     st_shared_v4(blk + static_cast<uint32_t>(row) * 128u + (static_cast<uint32_t>(c16 ^ (row & 7)) << 4),

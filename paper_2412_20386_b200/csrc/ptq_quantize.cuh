@@ -125,6 +125,48 @@ __device__ __forceinline__ bool quantize8_screen(uint32_t x0, uint32_t x1, uint3
     return worst > (kAsym ? kScreenThresholdAsym : kScreenThreshold);
 }
 
+// max(a, |b|, |c|) in one instruction (three-input max of sm_100); NaN operands are dropped like fmaxf does.
+__device__ __forceinline__ float max3_abs(float a, float b, float c)
+{
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(fabsf(b)), "f"(fabsf(c)));
+    return r;
+}
+
+// First-level route for signed codes, without any float-to-integer conversion instruction (those run
+// at a quarter of the rate of the other arithmetic here).  t = v' + 1.5*2^23 holds rint(v'), ties to
+// even, in its low mantissa bits, so for |v'| <= 127.25 the low BYTE of t is the two's-complement code;
+// the same t gives the tie distance.  Arithmetic is done two lanes per instruction (packed binary32
+// multiply / add / fma of sm_100; each lane is the ordinary correctly rounded operation).  Returns true
+// when the chunk has to go to the slower routes: a value within the tie band, a magnitude above
+// 127.25 (saturation is not handled here), or a NaN / infinity (their distance d is NaN, which the
+// sum below keeps while the maxima drop it).
+__device__ __forceinline__ bool quantize8_magic(uint32_t x0, uint32_t x1, uint32_t x2, uint32_t x3,
+                                                const float (&c8)[8], uint32_t &lo, uint32_t &hi)
+{
+    const uint32_t xw[4] = {x0, x1, x2, x3};
+    uint32_t tb[8];
+    float worst = 0.0f, big = 0.0f;
+    float2 nan_acc = make_float2(0.0f, 0.0f);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&xw[i]));
+        const float2 v = __fmul2_rn(f, make_float2(c8[2 * i], c8[2 * i + 1]));
+        const float2 t = __fadd2_rn(v, make_float2(kRoundMagic, kRoundMagic));
+        const float2 r = __fadd2_rn(t, make_float2(-kRoundMagic, -kRoundMagic));
+        const float2 d = __ffma2_rn(v, make_float2(-1.0f, -1.0f), r);      // rint(v) - v: exact, or NaN
+        nan_acc = __fadd2_rn(nan_acc, d);
+        worst = max3_abs(worst, d.x, d.y);
+        big = max3_abs(big, v.x, v.y);
+        tb[2 * i] = __float_as_uint(t.x);
+        tb[2 * i + 1] = __float_as_uint(t.y);
+    }
+    lo = pack4(static_cast<int>(tb[0]), static_cast<int>(tb[1]), static_cast<int>(tb[2]), static_cast<int>(tb[3]));
+    hi = pack4(static_cast<int>(tb[4]), static_cast<int>(tb[5]), static_cast<int>(tb[6]), static_cast<int>(tb[7]));
+    const float n = __fadd_rn(nan_acc.x, nan_acc.y);
+    return !(worst <= kScreenThreshold && big <= 127.25f && n == n);
+}
+
 // Exact route for the same 8 channels: two correctly rounded divisions per element.  s8 / rs8 point
 // at the channels' s and RN(1/s) in global memory.
 template <bool kFast, bool kAsym = false>
@@ -168,11 +210,37 @@ struct QuantParams {
 #ifndef PTQ_QUANT_CTAS_PER_SM
 #define PTQ_QUANT_CTAS_PER_SM 4
 #endif
-#ifndef PTQ_QUANT_IMGS_PER_TRIP
-#define PTQ_QUANT_IMGS_PER_TRIP 2
+#ifndef PTQ_QUANT_RING_DEPTH
+#define PTQ_QUANT_RING_DEPTH 4
 #endif
-constexpr int kQuantCtasPerSm = PTQ_QUANT_CTAS_PER_SM;     // resident CTAs per SM the vector kernel is built and launched for
-constexpr int kQuantImgsPerTrip = PTQ_QUANT_IMGS_PER_TRIP; // 16-byte loads per thread and trip (twice that in flight with the prefetch)
+constexpr int kQuantCtasPerSm = PTQ_QUANT_CTAS_PER_SM;   // resident CTAs per SM the vector kernel is built and launched for
+constexpr int kQuantRingDepth = PTQ_QUANT_RING_DEPTH;    // 16-byte loads in flight per thread
+
+__device__ __forceinline__ void cp_async_16(void *smem_dst, const void *gmem_src)
+{
+    const unsigned d = static_cast<unsigned>(__cvta_generic_to_shared(smem_dst));
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// The three routes for one chunk of 8 channels, cheapest first; every route that returns codes returns
+// the codes of the definition.
+template <bool kFast, bool kAsym>
+__device__ __forceinline__ uint2 quantize8(const uint4 &v, const float (&c8)[8], const float *s8, const float *rs8,
+                                           float dx, float rdx, int z)
+{
+    uint2 out;
+    bool exact = true;
+    if (kFast) {
+        bool slow = true;
+        if (!kAsym) slow = quantize8_magic(v.x, v.y, v.z, v.w, c8, out.x, out.y);
+        exact = slow && quantize8_screen<kAsym>(v.x, v.y, v.z, v.w, c8, out.x, out.y, z);
+    }
+    if (exact) quantize8_exact<kFast, kAsym>(v.x, v.y, v.z, v.w, s8, rs8, dx, rdx, out.x, out.y, z);
+    return out;
+}
 
 // Vector path: K % 8 == 0, x 16-byte aligned, q 8-byte aligned, q_pitch % 8 == 0.
 // A "chunk" is 8 consecutive channels of one token row: one 16-byte load, one 8-byte store.
@@ -182,11 +250,15 @@ constexpr int kQuantImgsPerTrip = PTQ_QUANT_IMGS_PER_TRIP; // 16-byte loads per 
 // per-token steps buy: the 8 combined reciprocals RN(1/s[k]) * RN(1/dx[t]) are formed once and kept
 // in registers, and the per-element work is convert, multiply, round, tie test.  Consecutive lanes
 // take consecutive chunks, so warp-wide accesses are contiguous 512-byte loads and 256-byte stores.
-// Each trip converts kQuantImgsPerTrip chunks and issues the next trip's loads first.
+// The loads are asynchronous copies (cp.async, L2 only) into a per-thread ring of shared-memory
+// slots, kQuantRingDepth images ahead.  A thread reads back only the slots it filled itself, so no
+// barrier is involved: cp.async.wait_group orders the thread's own copies.  Loads in flight hold no
+// registers, and their number does not depend on how far the arithmetic of the current chunk has got.
 template <bool kFast, bool kAsym = false>
 __global__ void __launch_bounds__(256, kQuantCtasPerSm) ptq_quantize_vec8_kernel(QuantParams p)
 {
-    constexpr int U = kQuantImgsPerTrip;
+    constexpr int D = kQuantRingDepth;
+    __shared__ uint4 ring[D][256];
     const int cpr = p.K >> 3;                                        // chunks per row
     const int cpi = p.T * cpr;                                       // chunks per image
     const long long gtid = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
@@ -214,34 +286,26 @@ __global__ void __launch_bounds__(256, kQuantCtasPerSm) ptq_quantize_vec8_kernel
     int8_t *qp = p.q + b * q_img + static_cast<long long>(t) * p.q_pitch + kc * 8;
     const long long x_step = S * x_img, q_step = S * q_img;
 
-    uint4 cur[U], nxt[U];
-    auto load_trip = [&](int b0, const __half *src, uint4 (&v)[U]) {
+    // fill the ring: slot i holds image b + i*S (one commit group per slot, empty past the last image)
 #pragma unroll
-        for (int j = 0; j < U; ++j) {
-            v[j] = make_uint4(0, 0, 0, 0);
-            if (b0 + j * S < p.B) v[j] = __ldcs(reinterpret_cast<const uint4 *>(src + j * x_step));
-        }
-    };
-    load_trip(b, xp, cur);
-    while (b < p.B) {
-        load_trip(b + U * S, xp + U * x_step, nxt);
-#pragma unroll
-        for (int j = 0; j < U; ++j) {
-            if (b + j * S < p.B) {
-                uint2 out;
-                bool exact = !kFast;
-                if (kFast) exact = quantize8_screen<kAsym>(cur[j].x, cur[j].y, cur[j].z, cur[j].w, c8, out.x, out.y, z);
-                if (exact)
-                    quantize8_exact<kFast, kAsym>(cur[j].x, cur[j].y, cur[j].z, cur[j].w, s8, rs8, d.x, d.y, out.x, out.y, z);
-                *reinterpret_cast<uint2 *>(qp + j * q_step) = out;
-            }
-        }
-#pragma unroll
-        for (int j = 0; j < U; ++j) cur[j] = nxt[j];
-        b += U * S;
-        xp += U * x_step;
-        qp += U * q_step;
+    for (int i = 0; i < D; ++i) {
+        if (b + i * S < p.B) cp_async_16(&ring[i][threadIdx.x], xp + i * x_step);
+        cp_async_commit();
     }
+    int slot = 0;
+    while (b < p.B) {
+        cp_async_wait<D - 1>();                                   // the oldest group, i.e. this slot, has landed
+        const uint4 v = ring[slot][threadIdx.x];
+        *reinterpret_cast<uint2 *>(qp) = quantize8<kFast, kAsym>(v, c8, s8, rs8, d.x, d.y, z);
+        // refill the slot just consumed (its value has been used above) with the image D*S further on
+        if (b + D * S < p.B) cp_async_16(&ring[slot][threadIdx.x], xp + D * x_step);
+        cp_async_commit();
+        slot = (slot + 1 == D) ? 0 : slot + 1;
+        b += S;
+        xp += x_step;
+        qp += q_step;
+    }
+    cp_async_wait<0>();
 }
 
 // Generic path: any K, any alignment; one element per thread per step.

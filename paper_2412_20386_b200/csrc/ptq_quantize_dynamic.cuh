@@ -139,18 +139,14 @@ __global__ void __launch_bounds__(256, PTQ_DYN_CTAS_PER_SM) ptq_quantize_dynamic
                 if (j < rows) {
                     const uint4 v = xrow[j][c];
                     uint2 out;
-                    bool exact = true;
                     if (fast_row[j]) {
                         const float c8[8] = {__fmul_rn(r0.x, rdx[j]), __fmul_rn(r0.y, rdx[j]), __fmul_rn(r0.z, rdx[j]),
                                              __fmul_rn(r0.w, rdx[j]), __fmul_rn(r1.x, rdx[j]), __fmul_rn(r1.y, rdx[j]),
                                              __fmul_rn(r1.z, rdx[j]), __fmul_rn(r1.w, rdx[j])};
-                        exact = quantize8_screen<false>(v.x, v.y, v.z, v.w, c8, out.x, out.y);
-                    }
-                    if (exact) {
-                        if (fast_row[j])
-                            quantize8_exact<true, false>(v.x, v.y, v.z, v.w, p.s + c * 8, p.rs + c * 8, dxr[j], rdx[j], out.x, out.y);
-                        else
-                            quantize8_exact<false, false>(v.x, v.y, v.z, v.w, p.s + c * 8, p.rs + c * 8, dxr[j], rdx[j], out.x, out.y);
+                        out = quantize8<true, false>(v, c8, p.s + c * 8, p.rs + c * 8, dxr[j], rdx[j], 0);
+                    } else {
+                        const float none[8] = {};
+                        out = quantize8<false, false>(v, none, p.s + c * 8, p.rs + c * 8, dxr[j], rdx[j], 0);
                     }
                     *reinterpret_cast<uint2 *>(p.q + (m0 + j) * p.q_pitch + c * 8) = out;
                 }
