@@ -462,8 +462,8 @@ def run_ours(args, specs, rank, world, local_rank):
 TRAFFIC = {
     ("ptq_gemm_dequant_kernel", "c3", "in_proj"): 41.175296e6 + 255.838976e6,
     ("ptq_gemm_dequant_kernel", "c3", "out_proj"): 78.698240e6 + 34.846976e6,
-    ("ptq_quantize_kernel", "c3", "in_proj"): 77.490688e6 + 6.991104e6,
-    ("ptq_quantize_kernel", "c3", "out_proj"): 154.978560e6 + 24.388096e6,
+    ("ptq_quantize_kernel", "c3", "in_proj"): 77.514752e6 + 10.142720e6,
+    ("ptq_quantize_kernel", "c3", "out_proj"): 155.153664e6 + 47.354624e6,
 }
 
 
