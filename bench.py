@@ -8,7 +8,8 @@ seeded synthetic activations, through the C ABI (`ptq_linear_forward`).  Prints 
 
   value          INT8 TOPS = sum_layers 2 M K N / step time, inputs resident in HBM, CUDA events
   e2e            the same metric with pinned HOST buffers: host->device copy of x, forward,
-                 device->host copy of y, all inside the timed region
+                 device->host copy of y, every step, all inside the timed region (the three stages
+                 run on three streams, double buffered, so copies and kernels overlap)
   roofline       the dominant kernel (largest share of the step), timed alone with CUDA events on
                  the launching stream in the same process; plus `kernels` with every kernel's figure
   cpu_baseline   the CPU oracle, as it stands, on a bounded row sample of the same workload
@@ -280,21 +281,54 @@ def run_ours(args, specs, rank, world, local_rank):
     step_ops = sum(layer_ops(d["spec"], d["spec"].B) for d in layers)
     touched = sum(d["x"].numel() * 2 + d["y"].numel() * 2 for d in layers)
 
-    def forward(d):
+    def forward(d, x=None, y=None):
+        x = d["x"] if x is None else x
+        y = d["y"] if y is None else y
         if args.scheme == "dynamic":
-            d["layer"].forward_dynamic(d["x"], y=d["y"], workspace=d["ws"])
+            d["layer"].forward_dynamic(x, y=y, workspace=d["ws"])
         else:
-            d["layer"].forward(d["x"], y=d["y"], workspace=d["ws"], flags=flags)
+            d["layer"].forward(x, y=y, workspace=d["ws"], flags=flags)
 
     def step():
         for d in layers:
             forward(d)
 
+    # End to end: every step copies every layer's x from pinned host memory and every y back to it.
+    # The three stages run on three streams with two device buffers per tensor, so the copy-in of the
+    # next item, the kernels of this one and the copy-out of the previous one overlap (PCIe is full
+    # duplex); events order each buffer's reuse.
+    comp = torch.cuda.current_stream()
+    s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+    for d in layers:
+        d["xb"] = [d["x"], torch.empty_like(d["x"])]
+        d["yb"] = [d["y"], torch.empty_like(d["y"])]
+        d["ev_in"] = [torch.cuda.Event(), torch.cuda.Event()]
+        d["ev_comp"] = [torch.cuda.Event(), torch.cuda.Event()]
+        d["ev_out"] = [torch.cuda.Event(), torch.cuda.Event()]
+        d["n"] = 0
+
     def step_e2e():
         for d in layers:
-            d["x"].copy_(d["x_host"], non_blocking=True)
-            forward(d)
-            d["y_host"].copy_(d["y"], non_blocking=True)
+            j, first = d["n"] & 1, d["n"] < 2
+            d["n"] += 1
+            with torch.cuda.stream(s_in):
+                if not first:
+                    s_in.wait_event(d["ev_comp"][j])          # the forward that last read this x buffer
+                d["xb"][j].copy_(d["x_host"], non_blocking=True)
+                d["ev_in"][j].record(s_in)
+            comp.wait_event(d["ev_in"][j])
+            if not first:
+                comp.wait_event(d["ev_out"][j])               # the copy-out that last read this y buffer
+            forward(d, d["xb"][j], d["yb"][j])
+            d["ev_comp"][j].record(comp)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(d["ev_comp"][j])
+                d["y_host"].copy_(d["yb"][j], non_blocking=True)
+                d["ev_out"][j].record(s_out)
+
+    def drain_e2e():
+        comp.wait_stream(s_in)
+        comp.wait_stream(s_out)
 
     def barrier():
         if world > 1:
@@ -341,12 +375,14 @@ def run_ours(args, specs, rank, world, local_rank):
     # ---- end to end with host buffers -------------------------------------------------------
     for _ in range(min(args.warmup, 3)):
         step_e2e()
+    drain_e2e()
     barrier()
     e2e_steps = max(3, min(args.steps, 20))
     f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     f0.record()
     for _ in range(e2e_steps):
         step_e2e()
+    drain_e2e()                                   # the last copy-out is inside the timed region
     f1.record()
     barrier()
     ms_e2e = f0.elapsed_time(f1) / e2e_steps
