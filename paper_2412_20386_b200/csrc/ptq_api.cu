@@ -964,17 +964,17 @@ static ptq_status_t calibrate_impl(int K, int N, int T, const void *xcal_fp16, i
     PTQ_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
     const long long M = static_cast<long long>(Bc) * T;
 
-    unsigned *d_bits = nullptr;   // [K] maxX bits, then [T] mu (or hi) bits, then [T] -lo bits
+    unsigned *d_bits = nullptr;   // [K] maxX bits, then [T] mu (or hi) bits, then [T] -lo bits, then [K] maxW bits
     float *d_out = nullptr;       // [K] s, then [T] dx, then [T] z (int)
     float *d_dw = nullptr;
     int8_t *d_w = nullptr;
     ptq_status_t st = PTQ_OK;
     auto body = [&]() -> ptq_status_t {
-        PTQ_CUDA(cudaMalloc(reinterpret_cast<void **>(&d_bits), sizeof(unsigned) * (K + 2 * T)));
+        PTQ_CUDA(cudaMalloc(reinterpret_cast<void **>(&d_bits), sizeof(unsigned) * (2 * K + 2 * T)));
         PTQ_CUDA(cudaMalloc(reinterpret_cast<void **>(&d_out), sizeof(float) * (K + 2 * T)));
         PTQ_CUDA(cudaMalloc(reinterpret_cast<void **>(&d_dw), sizeof(float) * N));
         PTQ_CUDA(cudaMalloc(reinterpret_cast<void **>(&d_w), static_cast<size_t>(N) * K));
-        PTQ_CUDA(cudaMemsetAsync(d_bits, 0, sizeof(unsigned) * (K + 2 * T), s));
+        PTQ_CUDA(cudaMemsetAsync(d_bits, 0, sizeof(unsigned) * (2 * K + 2 * T), s));
         PTQ_CUDA(cudaMemcpyAsync(d_dw, w_step, sizeof(float) * N, cudaMemcpyHostToDevice, s));
         PTQ_CUDA(cudaMemcpyAsync(d_w, w_q, static_cast<size_t>(N) * K, cudaMemcpyHostToDevice, s));
         const __half *x = static_cast<const __half *>(xcal_fp16);
@@ -982,7 +982,11 @@ static ptq_status_t calibrate_impl(int K, int N, int T, const void *xcal_fp16, i
         if (want > sms * 8ll) want = sms * 8ll;
         const int grid = static_cast<int>(want < 1 ? 1 : want);
         ptq::ptq_calib_colmax_kernel<<<grid, 256, 0, s>>>(x, M, K, d_bits);
-        ptq::ptq_calib_smooth_kernel<<<(K + 127) / 128, 128, 0, s>>>(d_bits, d_w, d_dw, N, K, d_out);
+        unsigned *d_wbits = d_bits + K + 2 * T;
+        const dim3 wgrid(static_cast<unsigned>((K + 127) / 128),
+                         static_cast<unsigned>((N + ptq::kCalibRowsPerBlock - 1) / ptq::kCalibRowsPerBlock));
+        ptq::ptq_calib_wmax_kernel<<<wgrid, 128, 0, s>>>(d_w, d_dw, N, K, d_wbits);
+        ptq::ptq_calib_smooth_kernel<<<(K + 127) / 128, 128, 0, s>>>(d_bits, d_wbits, K, d_out);
         if (act_zero_out) {
             ptq::ptq_calib_rowrange_kernel<<<grid, 256, 0, s>>>(x, M, K, T, d_out, d_bits + K, d_bits + K + T);
             ptq::ptq_calib_step_asym_kernel<<<(T + 127) / 128, 128, 0, s>>>(d_bits + K, d_bits + K + T, T, d_out + K,
@@ -991,7 +995,7 @@ static ptq_status_t calibrate_impl(int K, int N, int T, const void *xcal_fp16, i
             ptq::ptq_calib_rowmax_kernel<<<grid, 256, 0, s>>>(x, M, K, T, d_out, d_bits + K);
             ptq::ptq_calib_step_kernel<<<(T + 127) / 128, 128, 0, s>>>(d_bits + K, T, d_out + K);
         }
-        g_launches.fetch_add(4, std::memory_order_relaxed);
+        g_launches.fetch_add(5, std::memory_order_relaxed);
         PTQ_CUDA(cudaGetLastError());
         PTQ_CUDA(cudaMemcpyAsync(smooth_out, d_out, sizeof(float) * K, cudaMemcpyDeviceToHost, s));
         PTQ_CUDA(cudaMemcpyAsync(act_step_out, d_out + K, sizeof(float) * T, cudaMemcpyDeviceToHost, s));

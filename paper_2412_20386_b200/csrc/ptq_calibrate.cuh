@@ -54,20 +54,33 @@ __global__ void __launch_bounds__(256) ptq_calib_colmax_kernel(const __half *x, 
     }
 }
 
-// s[k] from maxX[k] and the weights; one thread per channel.
-__global__ void __launch_bounds__(128) ptq_calib_smooth_kernel(const unsigned *max_x_bits, const int8_t *wq,
-                                                               const float *dw, int N, int K, float *s)
+// maxW[k] = max_n |Wq[n,k]| * dw[n]: grid (channel blocks, row blocks); a thread scans kCalibRowsPerBlock
+// weight rows of its channel (coalesced across the block's channels) and merges with one atomicMax.
+constexpr int kCalibRowsPerBlock = 32;
+
+__global__ void __launch_bounds__(128) ptq_calib_wmax_kernel(const int8_t *wq, const float *dw, int N, int K,
+                                                             unsigned *max_w_bits)
 {
     const int k = blockIdx.x * blockDim.x + threadIdx.x;
     if (k >= K) return;
+    const int n0 = blockIdx.y * kCalibRowsPerBlock;
+    const int n1 = min(N, n0 + kCalibRowsPerBlock);
     float mw = 0.0f;
-    for (int n = 0; n < N; ++n) {
-        const float a = __fmul_rn(fabsf(static_cast<float>(wq[static_cast<long long>(n) * K + k])), dw[n]);
+    for (int n = n0; n < n1; ++n) {
+        const float a = __fmul_rn(fabsf(static_cast<float>(wq[static_cast<long long>(n) * K + k])), __ldg(dw + n));
         mw = fmaxf(mw, a);
     }
-    float mx = __uint_as_float(max_x_bits[k]);
-    mx = fmaxf(mx, kCalibFloor);
-    mw = fmaxf(mw, kCalibFloor);
+    if (mw > 0.0f) atomicMax(max_w_bits + k, __float_as_uint(mw));
+}
+
+// s[k] from maxX[k] and maxW[k]; one thread per channel.
+__global__ void __launch_bounds__(128) ptq_calib_smooth_kernel(const unsigned *max_x_bits, const unsigned *max_w_bits,
+                                                               int K, float *s)
+{
+    const int k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= K) return;
+    const float mx = fmaxf(__uint_as_float(max_x_bits[k]), kCalibFloor);
+    const float mw = fmaxf(__uint_as_float(max_w_bits[k]), kCalibFloor);
     s[k] = __fsqrt_rn(__fdiv_rn(mx, mw));
 }
 
