@@ -61,6 +61,16 @@ def _bind(path: str) -> ctypes.CDLL:
                                            vp, vp, vp, vp, vp, vp, vp, vp]
     L.ptqo_calibrate.restype = None
     L.ptqo_calibrate.argtypes = [vp, c_int, c_int, c_int, vp, vp, c_int, vp, vp]
+    L.ptqo_quantize4_one.restype = ctypes.c_int8
+    L.ptqo_quantize4_one.argtypes = [ctypes.c_uint16, ctypes.c_float, ctypes.c_float]
+    L.ptqo_quantize4.restype = None
+    L.ptqo_quantize4.argtypes = [vp, c_long, c_int, c_int, vp, vp, vp]
+    L.ptqo_pack_int4.restype = None
+    L.ptqo_pack_int4.argtypes = [vp, c_long, c_int, vp]
+    L.ptqo_unpack_int4.restype = None
+    L.ptqo_unpack_int4.argtypes = [vp, c_long, c_int, vp]
+    L.ptqo_calibrate4.restype = None
+    L.ptqo_calibrate4.argtypes = [vp, c_int, c_int, c_int, vp, vp, c_int, vp, vp]
     L.ptqo_search_act_step.restype = None
     L.ptqo_search_act_step.argtypes = [vp, c_int, c_int, c_int, vp, vp, c_int, c_int, vp, vp, vp]
     L.ptqo_quantize_dynamic.restype = None
@@ -340,3 +350,63 @@ def search_act_step(xcal, s, base, n_grid=100, j_lo=20):
     dx = np.empty(T, np.float32)
     lib().ptqo_search_act_step(_p(xcal), Bc, T, K, _p(s), _p(base), n_grid, j_lo, _p(loss), _p(best), _p(dx))
     return dx, best, loss
+
+
+# --------------------------------------------------------------------------- #
+# 4-bit variant (W4A4): signed range [-8, 7], two values per byte              #
+# --------------------------------------------------------------------------- #
+def quantize4_one(x_bits: int, s: float, dx: float) -> int:
+    return int(lib().ptqo_quantize4_one(int(x_bits), float(s), float(dx)))
+
+
+def quantize4(x, T, s, dx):
+    """x fp16 [M,K] -> int8-held 4-bit codes [M,K] = clip(round((x/s)/dx[t]), -8, 7)."""
+    x = _c(x, np.float16)
+    M, K = x.shape
+    s = _c(s, np.float32)
+    dx = _c(dx, np.float32)
+    assert s.shape == (K,) and dx.shape == (T,)
+    q = np.empty((M, K), np.int8)
+    lib().ptqo_quantize4(_p(x), M, K, T, _p(s), _p(dx), _p(q))
+    return q
+
+
+def pack_int4(d):
+    """int8 [rows, cols] with values in [-8, 7] -> uint8 [rows, (cols+1)//2], low nibble = even index."""
+    d = _c(d, np.int8)
+    rows, cols = d.shape
+    out = np.empty((rows, (cols + 1) // 2), np.uint8)
+    lib().ptqo_pack_int4(_p(d), rows, cols, _p(out))
+    return out
+
+
+def unpack_int4(packed, cols):
+    packed = _c(packed, np.uint8)
+    rows = packed.shape[0]
+    assert packed.shape[1] == (cols + 1) // 2
+    out = np.empty((rows, cols), np.int8)
+    lib().ptqo_unpack_int4(_p(packed), rows, cols, _p(out))
+    return out
+
+
+def calibrate4(xcal, wq, dw):
+    """Min-max calibration for 4-bit activations: (s fp32 [K], dx fp32 [T]) with dx = max|x/s| / 7."""
+    xcal = _c(xcal, np.float16)
+    Bc, T, K = xcal.shape
+    wq = _c(wq, np.int8)
+    N = wq.shape[0]
+    assert wq.shape == (N, K)
+    dw = _c(dw, np.float32)
+    s = np.empty(K, np.float32)
+    dx = np.empty(T, np.float32)
+    lib().ptqo_calibrate4(_p(xcal), Bc, T, K, _p(wq), _p(dw), N, _p(s), _p(dx))
+    return s, dx
+
+
+def linear_forward4(x, T, wq4, dw, s, dx, bias=None, taps=False):
+    """W4A4 end to end: 4-bit codes, contraction with the 4-bit weights (held one per int8), dequantization."""
+    x = _c(x, np.float16)
+    q = quantize4(x, T, s, dx)
+    acc = int_matmul(q, wq4)
+    y = dequant(acc, T, dx, dw, bias)
+    return (y, q, acc) if taps else y

@@ -496,3 +496,96 @@ void ptqo_search_act_step(const uint16_t *xcal, int Bc, int T, int K, const floa
         }
     }
 }
+
+/* ========================================================================= */
+/* 4-bit variant (W4A4 of the paper's latency table; Appendix B.1, part 2).   */
+/* Same quantizer with the signed 4-bit range:                                */
+/*   q4 = clip(round((x / s[k]) / dx[t]), -8, 7),   NaN -> 0, +-inf -> 7 / -8 */
+/* and the min-max step dx[t] = max(max|x/s|, 1e-5) / 7.  Two adjacent 4-bit  */
+/* values share a byte as the paper's packing step states: the value of even  */
+/* index in the low nibble, the next one in the high nibble,                  */
+/*   byte = (d[2i+1] << 4) | (d[2i] & 15);                                    */
+/* an odd-length row ends with a zero high nibble.  Unpacking sign-extends.   */
+/* The contraction and the dequantization are those of the 8-bit path.        */
+/* Pinned: hand-evaluated bytes of the packing formula (tests/golden);        */
+/* round trip over all nibble pairs; clip(q8) relation to the pinned 8-bit    */
+/* quantizer; numpy float32; no-clip invariant of the calibration.            */
+/* ========================================================================= */
+int8_t ptqo_quantize4_one(uint16_t x_half, float s, float dx)
+{
+    volatile float xf = ptqo_half_to_float(x_half);
+    volatile float u = xf / s;
+    volatile float v = u / dx;
+    float r;
+    if (isnan(v)) return 0;
+    r = nearbyintf(v);
+    if (r > 7.0f) r = 7.0f;
+    if (r < -8.0f) r = -8.0f;
+    return (int8_t)r;
+}
+
+void ptqo_quantize4(const uint16_t *x, long M, int K, int T, const float *s, const float *dx, int8_t *q)
+{
+    long m;
+#pragma omp parallel for schedule(static)
+    for (m = 0; m < M; ++m) {
+        int t = (int)(m % T);
+        int k;
+        for (k = 0; k < K; ++k)
+            q[m * K + k] = ptqo_quantize4_one(x[m * K + k], s[k], dx[t]);
+    }
+}
+
+/* rows of `cols` 4-bit values (each in [-8, 7], one per int8) -> rows of (cols + 1) / 2 bytes */
+void ptqo_pack_int4(const int8_t *d, long rows, int cols, uint8_t *packed)
+{
+    const int pb = (cols + 1) / 2;
+    long r;
+    for (r = 0; r < rows; ++r) {
+        int i;
+        for (i = 0; i < pb; ++i) {
+            int lo = d[r * cols + 2 * i];
+            int hi = (2 * i + 1 < cols) ? d[r * cols + 2 * i + 1] : 0;
+            packed[r * pb + i] = (uint8_t)(((hi << 4) | (lo & 15)) & 0xff);
+        }
+    }
+}
+
+void ptqo_unpack_int4(const uint8_t *packed, long rows, int cols, int8_t *d)
+{
+    const int pb = (cols + 1) / 2;
+    long r;
+    for (r = 0; r < rows; ++r) {
+        int k;
+        for (k = 0; k < cols; ++k) {
+            int nib = (packed[r * pb + k / 2] >> ((k & 1) * 4)) & 15;
+            d[r * cols + k] = (int8_t)(nib >= 8 ? nib - 16 : nib);
+        }
+    }
+}
+
+/* s[k] as in ptqo_calibrate (the weights are the unpacked 4-bit values); dx[t] = max(max|x/s|, floor) / 7 */
+void ptqo_calibrate4(const uint16_t *xcal, int Bc, int T, int K, const int8_t *wq, const float *dw, int N,
+                     float *s, float *dx)
+{
+    const float floor_ = 1e-5f;
+    int t;
+    ptqo_calibrate(xcal, Bc, T, K, wq, dw, N, s, dx);     /* s only; the 8-bit steps are replaced below */
+    for (t = 0; t < T; ++t) {
+        float mu = 0.0f;
+        int b, k;
+        for (b = 0; b < Bc; ++b) {
+            long m = (long)b * T + t;
+            for (k = 0; k < K; ++k) {
+                volatile float u = ptqo_half_to_float(xcal[m * K + k]) / s[k];
+                float a = fabsf(u);
+                if (a > mu) mu = a;
+            }
+        }
+        if (mu < floor_) mu = floor_;
+        {
+            volatile float d = mu / 7.0f;
+            dx[t] = d;
+        }
+    }
+}

@@ -9,6 +9,7 @@ import oracle
 import test_oracle_asym_pins as apins
 import test_oracle_pins as pins
 import test_oracle_search_pins as spins
+import test_oracle_int4_pins as ipins
 
 SRC = open(os.path.join(os.path.dirname(oracle.__file__), "ptq_oracle.c")).read()
 
@@ -90,6 +91,23 @@ MUTANTS = [
      [lambda: spins.test_search_matches_exact_rational_brute_force()]),
     ("search: returned step is the full step", "volatile float ratio = (float)best_j / (float)n_grid;", "volatile float ratio = 1.0f;",
      [lambda: spins.test_search_truncates_when_an_outlier_stretches_the_range()]),
+    ("int4: nibbles swapped when packing", "packed[r * pb + i] = (uint8_t)(((hi << 4) | (lo & 15)) & 0xff);",
+     "packed[r * pb + i] = (uint8_t)(((lo << 4) | (hi & 15)) & 0xff);",
+     [lambda: ipins.test_pack_matches_the_hand_evaluated_bytes()]),
+    ("int4: low nibble not masked", "packed[r * pb + i] = (uint8_t)(((hi << 4) | (lo & 15)) & 0xff);",
+     "packed[r * pb + i] = (uint8_t)(((hi << 4) | lo) & 0xff);",
+     [lambda: ipins.test_pack_matches_the_hand_evaluated_bytes()]),
+    ("int4: unpack without sign extension", "d[r * cols + k] = (int8_t)(nib >= 8 ? nib - 16 : nib);", "d[r * cols + k] = (int8_t)nib;",
+     [lambda: ipins.test_pack_round_trip_all_pairs_and_odd_lengths()]),
+    ("int4: unpack reads the wrong nibble", "int nib = (packed[r * pb + k / 2] >> ((k & 1) * 4)) & 15;",
+     "int nib = (packed[r * pb + k / 2] >> (((k & 1) ^ 1) * 4)) & 15;",
+     [lambda: ipins.test_pack_round_trip_all_pairs_and_odd_lengths()]),
+    ("int4: symmetric clamp", "if (r < -8.0f) r = -8.0f;", "if (r < -7.0f) r = -7.0f;",
+     [lambda: ipins.test_quantize4_is_the_clipped_eight_bit_code_and_matches_numpy()]),
+    ("int4: eight-bit clamp left in", "if (r > 7.0f) r = 7.0f;", "if (r > 127.0f) r = 127.0f;",
+     [lambda: ipins.test_quantize4_is_the_clipped_eight_bit_code_and_matches_numpy()]),
+    ("int4: step over 8 levels", "volatile float d = mu / 7.0f;", "volatile float d = mu / 8.0f;",
+     [lambda: ipins.test_calibrate4_steps_and_no_clip_invariant()]),
     ("dynamic step from the raw activations", "volatile float u = ptqo_half_to_float(x[m * K + k]) / s[k];\n            float a = fabsf(u);\n            if (a > mu) mu = a;                 /* NaN never wins the comparison */",
      "volatile float u = ptqo_half_to_float(x[m * K + k]);\n            float a = fabsf(u);\n            if (a > mu) mu = a;",
      [lambda: pins.test_dynamic_quantizer_vs_numpy_and_invariants()]),
