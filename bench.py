@@ -265,7 +265,15 @@ def run_ours(args, specs, rank, world, local_rank):
         x_host = torch.from_numpy(wl.activations(sp, wl.ROLE_EVAL)).pin_memory()
         wq, dw, bias = wl.weights(sp)
         xcal = torch.from_numpy(wl.activations(sp, wl.ROLE_CALIB)).to(dev)
-        if args.scheme == "pts-asym":
+        if args.scheme == "w4a4":
+            # 4-bit stand-ins for the workload's weights, packed two per byte (low nibble = even column)
+            w4 = np.clip(np.rint(wq.astype(np.float32) / 18.0), -8, 7).astype(np.int32)
+            if w4.shape[1] % 2:
+                w4 = np.concatenate([w4, np.zeros((w4.shape[0], 1), np.int32)], axis=1)
+            packed = (((w4[:, 1::2] << 4) | (w4[:, 0::2] & 15)) & 0xff).astype(np.uint8)
+            s, dx = ptq.calibrate_w4a4(xcal, packed, sp.K, dw)
+            layer = ptq.PtqLinear(packed, dw, s, dx, bias, packed4_K=sp.K)
+        elif args.scheme == "pts-asym":
             s, dx, z = ptq.calibrate_asym(xcal, wq, dw)          # Q0 on the GPU, with zero offsets
             layer = ptq.PtqLinear(wq, dw, s, dx, bias, act_zero=z)
         else:
@@ -513,9 +521,10 @@ def main():
     ap.add_argument("--path", default="unfused", choices=["unfused", "fused", "pair"],
                     help="unfused: quantize kernel + GEMM kernel (fastest at present, the default); "
                          "fused: PTQ_FLAG_FUSED_PROLOGUE; pair: PTQ_FLAG_CTA_PAIR")
-    ap.add_argument("--scheme", default="pts", choices=["pts", "pts-asym", "dynamic"],
+    ap.add_argument("--scheme", default="pts", choices=["pts", "pts-asym", "dynamic", "w4a4"],
                     help="pts: symmetric per-token-static codes (the default); pts-asym: with a zero offset per token "
-                         "position; dynamic: the per-token dynamic comparator (row steps measured at run time)")
+                         "position; dynamic: the per-token dynamic comparator (row steps measured at run time); "
+                         "w4a4: 4-bit codes and packed 4-bit weights on the 8-bit tensor-core path")
     ap.add_argument("--graph", action="store_true",
                     help="capture one step in a CUDA graph and time replays (for launch-bound workloads such as c1)")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)

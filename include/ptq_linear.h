@@ -231,6 +231,35 @@ ptq_status_t ptq_calibrate(int K, int N, int T, const void *xcal_fp16, int Bc,
                            float *smooth_out, float *act_step_out, void *stream);
 
 /*
+ * W4A4 layers (the bit width of the paper's latency table; Appendix B.1, quantization part).  The
+ * arithmetic is that of ptq_linear_create / ptq_linear_forward with the signed 4-bit range:
+ *     q = clamp(rne((x / s[k]) / act_step[t]), -8, 7),   acc = sum_k q * w4,   y as before,
+ * NaN -> 0, +inf -> 7, -inf -> -8.  Weights arrive packed two per byte as the paper states,
+ *     byte = (w[n, 2i+1] << 4) | (w[n, 2i] & 15)      (low nibble = even column, two's complement),
+ * rows of (K+1)/2 bytes, an odd K ending with an unused high nibble.  The integer tensor-core
+ * instruction of sm_100 takes 8-bit operands, so the library unpacks the weights once at create and
+ * keeps the activation codes one per byte in the workspace: 4-bit layers run at the speed of 8-bit
+ * ones and save only the bytes of the stored weights.  All other entry points (workspace_bytes,
+ * forward, forward_debug, quantize, gemm_dequant, forward_static) accept such a handle; the fused
+ * prologue and CTA-pair flags are ignored, the dynamic comparator is refused.
+ *   w_q_packed   host, [N, (K+1)/2] bytes
+ *   act_step     host, [T]; ptq_calibrate_w4a4 returns the min-max steps max|x/s| / 7
+ */
+ptq_status_t ptq_linear_create_w4a4(ptq_linear_t **out, int K, int N, int T, const uint8_t *w_q_packed,
+                                    const float *w_step, const float *smooth, const float *act_step,
+                                    const float *bias, unsigned flags);
+ptq_status_t ptq_calibrate_w4a4(int K, int N, int T, const void *xcal_fp16, int Bc, const uint8_t *w_q_packed,
+                                const float *w_step, float *smooth_out, float *act_step_out, void *stream);
+/*
+ * Q1 of a W4A4 layer with the codes packed two per byte exactly as the paper's quantization step
+ * writes them (byte = (q[m, 2i+1] << 4) | (q[m, 2i] & 15)), for storage or transport.
+ *   q_packed    device, [B*T, (K+1)/2] bytes
+ *   workspace   device, 16-byte aligned, at least ptq_linear_workspace_bytes(h, B, PTQ_FLAG_NONE) bytes
+ */
+ptq_status_t ptq_quantize_packed4(const ptq_linear_t *h, const void *x_fp16, int B, void *q_packed, void *workspace,
+                                  size_t workspace_bytes, void *stream);
+
+/*
  * Step-size search (Sec. 5.2, second stage; the "+Truncation" row of the ablation): for every token
  * position the candidate step
  *     Delta[t,j] = base_step[t] * (j / n_grid),   j = j_lo .. n_grid

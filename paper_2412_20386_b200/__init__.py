@@ -7,5 +7,5 @@ synthetic inputs (``workloads.py``).  The shared library is loaded on first use
 and the binding raises if it is missing: there is no CPU fallback.
 """
 from . import workloads  # noqa: F401
-from .binding import (PtqError, PtqLinear, calibrate, calibrate_asym, search_act_step, library_path, load_library,  # noqa: F401
+from .binding import (PtqError, PtqLinear, calibrate, calibrate_asym, calibrate_w4a4, search_act_step, library_path, load_library,  # noqa: F401
                       FLAG_FUSED_PROLOGUE, FLAG_CTA_PAIR)

@@ -82,6 +82,12 @@ def load_library() -> ctypes.CDLL:
     L.ptq_linear_forward_debug.argtypes = [vp, vp, ci, vp, vp, vp, vp, sz, cu, vp]
     L.ptq_calibrate.restype = ci
     L.ptq_calibrate.argtypes = [ci, ci, ci, vp, ci, vp, vp, vp, vp, vp]
+    L.ptq_linear_create_w4a4.restype = ci
+    L.ptq_linear_create_w4a4.argtypes = [ctypes.POINTER(vp), ci, ci, ci, vp, vp, vp, vp, vp, cu]
+    L.ptq_calibrate_w4a4.restype = ci
+    L.ptq_calibrate_w4a4.argtypes = [ci, ci, ci, vp, ci, vp, vp, vp, vp, vp]
+    L.ptq_quantize_packed4.restype = ci
+    L.ptq_quantize_packed4.argtypes = [vp, vp, ci, vp, vp, sz, vp]
     L.ptq_search_act_step.restype = ci
     L.ptq_search_act_step.argtypes = [ci, ci, vp, ci, vp, vp, ci, ci, vp, vp, vp, vp]
     L.ptq_linear_describe.restype = ci
@@ -130,12 +136,19 @@ def kernel_launch_count() -> int:
 class PtqLinear:
     """One PTS W8A8 linear layer on the current CUDA device (``ptq_linear_create``)."""
 
-    def __init__(self, w_q, w_step, smooth, act_step, bias=None, flags: int = 0, act_zero=None):
+    def __init__(self, w_q, w_step, smooth, act_step, bias=None, flags: int = 0, act_zero=None, packed4_K=None):
         L = load_library()
-        w_q = _host(w_q, np.int8)
-        if w_q.ndim != 2:
-            raise ValueError("w_q must be [N,K]")
-        self.N, self.K = int(w_q.shape[0]), int(w_q.shape[1])
+        self.w4a4 = packed4_K is not None
+        if self.w4a4:                                            # ``ptq_linear_create_w4a4``: w_q is [N, (K+1)//2] bytes
+            w_q = _host(w_q, np.uint8)
+            if w_q.ndim != 2 or w_q.shape[1] != (int(packed4_K) + 1) // 2:
+                raise ValueError("packed w_q must be [N, (K+1)//2] bytes")
+            self.N, self.K = int(w_q.shape[0]), int(packed4_K)
+        else:
+            w_q = _host(w_q, np.int8)
+            if w_q.ndim != 2:
+                raise ValueError("w_q must be [N,K]")
+            self.N, self.K = int(w_q.shape[0]), int(w_q.shape[1])
         act_step = _host(act_step, np.float32)
         self.T = int(act_step.shape[0])
         w_step = _host(w_step, np.float32, (self.N,))
@@ -143,7 +156,12 @@ class PtqLinear:
         bias = _host(bias, np.float32, (self.N,))
         h = ctypes.c_void_p()
         self.asym = act_zero is not None
-        if self.asym:                                            # ``ptq_linear_create_asym``: unsigned codes
+        if self.w4a4:
+            if self.asym:
+                raise ValueError("W4A4 layers are symmetric")
+            _check(L.ptq_linear_create_w4a4(ctypes.byref(h), self.K, self.N, self.T, _hp(w_q), _hp(w_step),
+                                            _hp(smooth), _hp(act_step), _hp(bias), flags))
+        elif self.asym:                                          # ``ptq_linear_create_asym``: unsigned codes
             act_zero = _host(act_zero, np.int32, (self.T,))
             _check(L.ptq_linear_create_asym(ctypes.byref(h), self.K, self.N, self.T, _hp(w_q), _hp(w_step),
                                             _hp(smooth), _hp(act_step), _hp(act_zero), _hp(bias), flags))
@@ -256,6 +274,17 @@ class PtqLinear:
         _check(self._L.ptq_quantize(self._h, x.data_ptr(), B, q.data_ptr(), _stream_ptr(stream)))
         return q
 
+    def quantize_packed4(self, x, stream=None):
+        """``ptq_quantize_packed4``: x fp16 [B,T,K] -> 4-bit codes packed two per byte, uint8 [B,T,(K+1)//2]."""
+        import torch
+        B = self._batch(x)
+        out = torch.empty((B, self.T, (self.K + 1) // 2), dtype=torch.uint8, device=x.device)
+        need = self.workspace_bytes(B, 0)
+        ws = torch.empty(need, dtype=torch.uint8, device=x.device)
+        _check(self._L.ptq_quantize_packed4(self._h, x.data_ptr(), B, out.data_ptr(), ws.data_ptr(), need,
+                                            _stream_ptr(stream)))
+        return out
+
     def code_pitch(self) -> int:
         return int(self._L.ptq_linear_code_pitch(self._h))
 
@@ -345,3 +374,22 @@ def search_act_step(xcal, smooth, base_step, n_grid: int = 100, j_lo: int = 20, 
                                  dx.ctypes.data, best.ctypes.data,
                                  loss.ctypes.data if loss is not None else None, _stream_ptr(stream)))
     return dx, best, loss
+
+
+def calibrate_w4a4(xcal, w_q_packed, K: int, w_step, stream=None):
+    """``ptq_calibrate_w4a4``: device fp16 [Bc,T,K], packed 4-bit weights -> (s fp32 [K], dx fp32 [T] = max|x/s|/7)."""
+    import torch
+    L = load_library()
+    if xcal.dtype != torch.float16 or not xcal.is_cuda or not xcal.is_contiguous() or xcal.dim() != 3 or xcal.shape[2] != K:
+        raise ValueError("xcal must be a contiguous CUDA float16 tensor [Bc,T,K]")
+    Bc, T = int(xcal.shape[0]), int(xcal.shape[1])
+    w_q_packed = _host(w_q_packed, np.uint8)
+    N = int(w_q_packed.shape[0])
+    if w_q_packed.shape != (N, (K + 1) // 2):
+        raise ValueError("packed w_q must be [N, (K+1)//2] bytes")
+    w_step = _host(w_step, np.float32, (N,))
+    s = np.empty(K, np.float32)
+    dx = np.empty(T, np.float32)
+    _check(L.ptq_calibrate_w4a4(K, N, T, xcal.data_ptr(), Bc, w_q_packed.ctypes.data, w_step.ctypes.data,
+                                s.ctypes.data, dx.ctypes.data, _stream_ptr(stream)))
+    return s, dx

@@ -117,6 +117,7 @@ struct ptq_linear {
     int *d_zp = nullptr;                                 // [T] zero offsets (asymmetric layers only)
     int *d_wsum = nullptr;                               // row sums of Wq, padded like d_dw (asymmetric only)
     bool asym = false;
+    int act_bits = 8;          // 8: codes in [-128,127] (or [0,255]); 4: codes in [-8,7], one per byte
     unsigned *d_status = nullptr;
     CUtensorMap tmW;
     CUtensorMap tmWh;          // same weights, box of BN/2 rows: the half tile one CTA of a pair loads
@@ -226,11 +227,16 @@ ptq_status_t launch_quantize(const ptq_linear *h, const void *x, long long M, vo
     p.imgs_per_iter = static_cast<int>(S);
     if (vec) {
         const int grid = static_cast<int>(S * cpi / 256);
-        if (h->asym) {
+        if (h->act_bits == 4) {
             if (h->fast_div)
-                ptq::ptq_quantize_vec8_kernel<true, true><<<grid, 256, 0, stream>>>(p);
+                ptq::ptq_quantize_vec8_kernel<true, ptq::kCodeS4><<<grid, 256, 0, stream>>>(p);
             else
-                ptq::ptq_quantize_vec8_kernel<false, true><<<grid, 256, 0, stream>>>(p);
+                ptq::ptq_quantize_vec8_kernel<false, ptq::kCodeS4><<<grid, 256, 0, stream>>>(p);
+        } else if (h->asym) {
+            if (h->fast_div)
+                ptq::ptq_quantize_vec8_kernel<true, ptq::kCodeU8><<<grid, 256, 0, stream>>>(p);
+            else
+                ptq::ptq_quantize_vec8_kernel<false, ptq::kCodeU8><<<grid, 256, 0, stream>>>(p);
         } else if (h->fast_div)
             ptq::ptq_quantize_vec8_kernel<true><<<grid, 256, 0, stream>>>(p);
         else
@@ -240,15 +246,21 @@ ptq_status_t launch_quantize(const ptq_linear *h, const void *x, long long M, vo
         const long long cap = static_cast<long long>(h->num_sms) * 8;
         if (want > cap) want = cap;
         if (want < 1) want = 1;
-        if (h->asym) {
+        const int g = static_cast<int>(want);
+        if (h->act_bits == 4) {
             if (h->fast_div)
-                ptq::ptq_quantize_scalar_kernel<true, true><<<static_cast<int>(want), 256, 0, stream>>>(p);
+                ptq::ptq_quantize_scalar_kernel<true, ptq::kCodeS4><<<g, 256, 0, stream>>>(p);
             else
-                ptq::ptq_quantize_scalar_kernel<false, true><<<static_cast<int>(want), 256, 0, stream>>>(p);
+                ptq::ptq_quantize_scalar_kernel<false, ptq::kCodeS4><<<g, 256, 0, stream>>>(p);
+        } else if (h->asym) {
+            if (h->fast_div)
+                ptq::ptq_quantize_scalar_kernel<true, ptq::kCodeU8><<<g, 256, 0, stream>>>(p);
+            else
+                ptq::ptq_quantize_scalar_kernel<false, ptq::kCodeU8><<<g, 256, 0, stream>>>(p);
         } else if (h->fast_div)
-            ptq::ptq_quantize_scalar_kernel<true><<<static_cast<int>(want), 256, 0, stream>>>(p);
+            ptq::ptq_quantize_scalar_kernel<true><<<g, 256, 0, stream>>>(p);
         else
-            ptq::ptq_quantize_scalar_kernel<false><<<static_cast<int>(want), 256, 0, stream>>>(p);
+            ptq::ptq_quantize_scalar_kernel<false><<<g, 256, 0, stream>>>(p);
     }
     g_launches.fetch_add(1, std::memory_order_relaxed);
     PTQ_CUDA(cudaGetLastError());
@@ -567,7 +579,7 @@ void ptq_linear_destroy(ptq_linear_t *h)
 
 static ptq_status_t create_impl(ptq_linear_t **out, int K, int N, int T, const int8_t *w_q, const float *w_step,
                                 const float *smooth, const float *act_step, const int32_t *act_zero,
-                                const float *bias, unsigned flags)
+                                const float *bias, unsigned flags, int act_bits = 8)
 {
     if (!out) return fail(PTQ_ERR_NULL, "out must not be NULL");
     *out = nullptr;
@@ -628,8 +640,9 @@ static ptq_status_t create_impl(ptq_linear_t **out, int K, int N, int T, const i
     h->last_mmas = (K - (h->k_blocks - 1) * ptq::kBK + 31) / 32;
 
     h->asym = act_zero != nullptr;
+    h->act_bits = act_bits;
     choose_astat(h);
-    if (h->asym) h->as_ok = false;          // asymmetric layers run the quantize kernel + single-CTA GEMM kernel only
+    if (h->asym || act_bits != 8) h->as_ok = false;   // these layers run the quantize kernel + single-CTA GEMM kernel only
     int Npad = h->n_tiles * h->BN;
     if (h->as_ok && h->as_n_tiles * h->as_BN > Npad) Npad = h->as_n_tiles * h->as_BN;
     const int Nvec = round_up(Npad, 64) + 64;
@@ -740,7 +753,7 @@ int ptq_linear_describe(const ptq_linear_t *h, char *buf, int buf_bytes)
     const int n = snprintf(tmp, sizeof(tmp),
                            "K=%d N=%d T=%d Kpad=%d%s | quantize: %s | gemm: BN=%d n_tiles=%d k_blocks=%d "
                            "pair_clusters=%d | fused: %s BN=%d n_tiles=%d w_stages=%d staging=%d smem=%d",
-                           h->K, h->N, h->T, h->Kpad, h->asym ? " asymmetric" : "",
+                           h->K, h->N, h->T, h->Kpad, h->asym ? " asymmetric" : (h->act_bits == 4 ? " w4a4" : ""),
                            h->fast_div ? "screened reciprocal route" : "IEEE division",
                            h->BN, h->n_tiles, h->k_blocks, h->max_pairs,
                            (h->as_ok && h->K % 16 == 0) ? "yes" : "no", h->as_BN, h->as_n_tiles, h->as_w_stages,
@@ -903,7 +916,8 @@ ptq_status_t ptq_linear_forward_dynamic_debug(const ptq_linear_t *h, const void 
 {
     ptq_status_t st = validate_forward(h, x_fp16, B, y_fp16);
     if (st != PTQ_OK) return st;
-    if (h->asym) return fail(PTQ_ERR_VALUE, "the dynamic comparator is defined for symmetric layers only");
+    if (h->asym || h->act_bits != 8)
+        return fail(PTQ_ERR_VALUE, "the dynamic comparator is defined for symmetric 8-bit layers only");
     const long long M = static_cast<long long>(B) * h->T;
     const size_t codes = dynamic_codes_bytes(h, M);
     const size_t need = codes + static_cast<size_t>(M) * sizeof(float);
@@ -951,7 +965,7 @@ ptq_status_t ptq_linear_device_status(const ptq_linear_t *h)
 
 static ptq_status_t calibrate_impl(int K, int N, int T, const void *xcal_fp16, int Bc, const int8_t *w_q,
                                    const float *w_step, float *smooth_out, float *act_step_out,
-                                   int32_t *act_zero_out, void *stream)
+                                   int32_t *act_zero_out, void *stream, float qmax = 127.0f)
 {
     if (!xcal_fp16 || !w_q || !w_step || !smooth_out || !act_step_out)
         return fail(PTQ_ERR_NULL, "calibrate: pointers must not be NULL");
@@ -993,7 +1007,7 @@ static ptq_status_t calibrate_impl(int K, int N, int T, const void *xcal_fp16, i
                                                                            reinterpret_cast<int *>(d_out + K + T));
         } else {
             ptq::ptq_calib_rowmax_kernel<<<grid, 256, 0, s>>>(x, M, K, T, d_out, d_bits + K);
-            ptq::ptq_calib_step_kernel<<<(T + 127) / 128, 128, 0, s>>>(d_bits + K, T, d_out + K);
+            ptq::ptq_calib_step_kernel<<<(T + 127) / 128, 128, 0, s>>>(d_bits + K, T, d_out + K, qmax);
         }
         g_launches.fetch_add(5, std::memory_order_relaxed);
         PTQ_CUDA(cudaGetLastError());
@@ -1024,6 +1038,73 @@ ptq_status_t ptq_calibrate_asym(int K, int N, int T, const void *xcal_fp16, int 
 {
     if (!act_zero_out) return fail(PTQ_ERR_NULL, "calibrate: pointers must not be NULL");
     return calibrate_impl(K, N, T, xcal_fp16, Bc, w_q, w_step, smooth_out, act_step_out, act_zero_out, stream);
+}
+
+// Sign-extending unpack of rows of 4-bit values, two per byte, low nibble = even column.
+static void unpack_int4_host(const uint8_t *packed, int rows, int cols, std::vector<int8_t> &out)
+{
+    const int pb = (cols + 1) / 2;
+    out.resize(static_cast<size_t>(rows) * cols);
+    for (int r = 0; r < rows; ++r)
+        for (int k = 0; k < cols; ++k) {
+            const int nib = (packed[static_cast<size_t>(r) * pb + k / 2] >> ((k & 1) * 4)) & 15;
+            out[static_cast<size_t>(r) * cols + k] = static_cast<int8_t>(nib >= 8 ? nib - 16 : nib);
+        }
+}
+
+ptq_status_t ptq_linear_create_w4a4(ptq_linear_t **out, int K, int N, int T, const uint8_t *w_q_packed,
+                                    const float *w_step, const float *smooth, const float *act_step,
+                                    const float *bias, unsigned flags)
+{
+    if (!out) return fail(PTQ_ERR_NULL, "out must not be NULL");
+    *out = nullptr;
+    if (!w_q_packed) return fail(PTQ_ERR_NULL, "w_q_packed must not be NULL");
+    if (K < 1 || K > PTQ_MAX_K || N < 1 || N > PTQ_MAX_N)
+        return fail(PTQ_ERR_SHAPE, "K, N out of range (K=%d N=%d)", K, N);
+    std::vector<int8_t> w;
+    unpack_int4_host(w_q_packed, N, K, w);
+    return create_impl(out, K, N, T, w.data(), w_step, smooth, act_step, nullptr, bias, flags, 4);
+}
+
+ptq_status_t ptq_calibrate_w4a4(int K, int N, int T, const void *xcal_fp16, int Bc, const uint8_t *w_q_packed,
+                                const float *w_step, float *smooth_out, float *act_step_out, void *stream)
+{
+    if (!w_q_packed) return fail(PTQ_ERR_NULL, "calibrate: pointers must not be NULL");
+    if (K < 1 || K > PTQ_MAX_K || N < 1 || N > PTQ_MAX_N)
+        return fail(PTQ_ERR_SHAPE, "calibrate: dimensions out of range (K=%d N=%d)", K, N);
+    std::vector<int8_t> w;
+    unpack_int4_host(w_q_packed, N, K, w);
+    return calibrate_impl(K, N, T, xcal_fp16, Bc, w.data(), w_step, smooth_out, act_step_out, nullptr, stream, 7.0f);
+}
+
+ptq_status_t ptq_quantize_packed4(const ptq_linear_t *h, const void *x_fp16, int B, void *q_packed, void *workspace,
+                                  size_t workspace_bytes, void *stream)
+{
+    if (!h || !x_fp16 || !q_packed || !workspace) return fail(PTQ_ERR_NULL, "handle, x, q and workspace must not be NULL");
+    if (h->act_bits != 4) return fail(PTQ_ERR_VALUE, "packed 4-bit codes need a layer made by ptq_linear_create_w4a4");
+    if (B < 1) return fail(PTQ_ERR_SHAPE, "B must be >= 1 (got %d)", B);
+    if (reinterpret_cast<uintptr_t>(x_fp16) % 2) return fail(PTQ_ERR_ALIGN, "x must be 2-byte aligned");
+    if (reinterpret_cast<uintptr_t>(workspace) % 16) return fail(PTQ_ERR_ALIGN, "workspace must be 16-byte aligned");
+    ptq_status_t st = check_device(h);
+    if (st != PTQ_OK) return st;
+    const long long M = static_cast<long long>(B) * h->T;
+    const size_t need = static_cast<size_t>(M) * h->Kpad;
+    if (workspace_bytes < need) return fail(PTQ_ERR_SHAPE, "workspace has %zu bytes, %zu needed", workspace_bytes, need);
+    const size_t out_bytes = static_cast<size_t>(M) * ((h->K + 1) / 2);
+    if (ranges_overlap(workspace, need, q_packed, out_bytes) ||
+        ranges_overlap(workspace, need, x_fp16, static_cast<size_t>(M) * h->K * 2) ||
+        ranges_overlap(q_packed, out_bytes, x_fp16, static_cast<size_t>(M) * h->K * 2))
+        return fail(PTQ_ERR_VALUE, "x, q and workspace overlap");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if ((st = launch_quantize(h, x_fp16, M, workspace, h->Kpad, s)) != PTQ_OK) return st;
+    long long want = (static_cast<long long>(out_bytes) + 255) / 256;
+    const long long cap = static_cast<long long>(h->num_sms) * 16;
+    if (want > cap) want = cap;
+    ptq::ptq_pack_int4_kernel<<<static_cast<int>(want), 256, 0, s>>>(static_cast<const int8_t *>(workspace), M, h->K,
+                                                                    h->Kpad, static_cast<uint8_t *>(q_packed));
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    PTQ_CUDA(cudaGetLastError());
+    return PTQ_OK;
 }
 
 }  // extern "C"

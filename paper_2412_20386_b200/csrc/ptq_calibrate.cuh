@@ -102,11 +102,11 @@ __global__ void __launch_bounds__(256) ptq_calib_rowmax_kernel(const __half *x, 
     }
 }
 
-__global__ void __launch_bounds__(128) ptq_calib_step_kernel(const unsigned *mu_bits, int T, float *dx)
+__global__ void __launch_bounds__(128) ptq_calib_step_kernel(const unsigned *mu_bits, int T, float *dx, float qmax)
 {
     const int t = blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= T) return;
-    dx[t] = __fdiv_rn(fmaxf(__uint_as_float(mu_bits[t]), kCalibFloor), 127.0f);
+    dx[t] = __fdiv_rn(fmaxf(__uint_as_float(mu_bits[t]), kCalibFloor), qmax);      // 127 levels, or 7 for 4-bit codes
 }
 
 // --- asymmetric variant: per-token-position range [lo, hi] of x/s, always containing zero ----------

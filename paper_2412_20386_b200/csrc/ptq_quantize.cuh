@@ -46,25 +46,31 @@ __device__ __forceinline__ int f32_to_code_asym(float v, int z)
     return min(max(static_cast<int>(r) + z, 0), 255);
 }
 
-template <bool kAsym>
+// Code formats: signed 8-bit (the path of Sec. 5.1), unsigned 8-bit with a zero offset, signed 4-bit
+// held one per byte (W4A4 of the latency table: clip to [-8, 7]).
+constexpr int kCodeS8 = 0, kCodeU8 = 1, kCodeS4 = 2;
+
+template <int kMode>
 __device__ __forceinline__ int code_of(float v, int z)
 {
-    return kAsym ? f32_to_code_asym(v, z) : f32_to_code(v);
+    if (kMode == kCodeU8) return f32_to_code_asym(v, z);
+    const int r = f32_to_code(v);
+    return kMode == kCodeS4 ? min(max(r, -8), 7) : r;
 }
 
 // One element, IEEE divisions (any positive finite s, dx; also the path for inf/NaN inputs).
-template <bool kAsym = false>
+template <int kMode = kCodeS8>
 __device__ __forceinline__ int quantize_ieee(float xf, float s, float dx, int z = 0)
 {
-    return code_of<kAsym>(__fdiv_rn(__fdiv_rn(xf, s), dx), z);
+    return code_of<kMode>(__fdiv_rn(__fdiv_rn(xf, s), dx), z);
 }
 
 // One element through the reciprocal route (finite xf, scales inside the safe range).
-template <bool kAsym = false>
+template <int kMode = kCodeS8>
 __device__ __forceinline__ int quantize_fast(float xf, float s, float rs, float dx, float rdx, int z = 0)
 {
     const float u = div_rn_by_reciprocal(xf, s, rs);
-    return code_of<kAsym>(div_rn_by_reciprocal(u, dx, rdx), z);
+    return code_of<kMode>(div_rn_by_reciprocal(u, dx, rdx), z);
 }
 
 __device__ __forceinline__ uint32_t pack4(int a, int b, int c, int d)
@@ -100,9 +106,9 @@ __device__ __forceinline__ float dist_to_integer(float v)
 // infinities saturate on both routes, so whether such values pass the test or not only costs time:
 // the final codes are always those of the definition.
 // Valid only when every scale lies in [2^-30, 2^30] (no under/overflow in c or x * c).
-// kAsym: the codes are clip(rint(v') + z, 0, 255); ties of v' are still the only place where v' and v
+// Unsigned codes: clip(rint(v') + z, 0, 255); ties of v' are still the only place where v' and v
 // can disagree, with the wider band of kScreenThresholdAsym.
-template <bool kAsym = false>
+template <int kMode = kCodeS8>
 __device__ __forceinline__ bool quantize8_screen(uint32_t x0, uint32_t x1, uint32_t x2, uint32_t x3,
                                                  const float (&c8)[8], uint32_t &lo, uint32_t &hi, int z = 0)
 {
@@ -116,13 +122,13 @@ __device__ __forceinline__ bool quantize8_screen(uint32_t x0, uint32_t x1, uint3
         const float2 f = __half22float2(h);
         const float v0 = __fmul_rn(f.x, c8[2 * i]);
         const float v1 = __fmul_rn(f.y, c8[2 * i + 1]);
-        c[2 * i] = code_of<kAsym>(v0, z);
-        c[2 * i + 1] = code_of<kAsym>(v1, z);
+        c[2 * i] = code_of<kMode>(v0, z);
+        c[2 * i + 1] = code_of<kMode>(v1, z);
         worst = fmaxf(worst, fmaxf(dist_to_integer(v0), dist_to_integer(v1)));
     }
     lo = pack4(c[0], c[1], c[2], c[3]);
     hi = pack4(c[4], c[5], c[6], c[7]);
-    return worst > (kAsym ? kScreenThresholdAsym : kScreenThreshold);
+    return worst > (kMode == kCodeU8 ? kScreenThresholdAsym : kScreenThreshold);
 }
 
 // max(a, |b|, |c|) in one instruction (three-input max of sm_100); NaN operands are dropped like fmaxf does.
@@ -141,6 +147,7 @@ __device__ __forceinline__ float max3_abs(float a, float b, float c)
 // when the chunk has to go to the slower routes: a value within the tie band, a magnitude above
 // 127.25 (saturation is not handled here), or a NaN / infinity (their distance d is NaN, which the
 // sum below keeps while the maxima drop it).
+template <int kMode = kCodeS8>
 __device__ __forceinline__ bool quantize8_magic(uint32_t x0, uint32_t x1, uint32_t x2, uint32_t x3,
                                                 const float (&c8)[8], uint32_t &lo, uint32_t &hi)
 {
@@ -164,12 +171,12 @@ __device__ __forceinline__ bool quantize8_magic(uint32_t x0, uint32_t x1, uint32
     lo = pack4(static_cast<int>(tb[0]), static_cast<int>(tb[1]), static_cast<int>(tb[2]), static_cast<int>(tb[3]));
     hi = pack4(static_cast<int>(tb[4]), static_cast<int>(tb[5]), static_cast<int>(tb[6]), static_cast<int>(tb[7]));
     const float n = __fadd_rn(nan_acc.x, nan_acc.y);
-    return !(worst <= kScreenThreshold && big <= 127.25f && n == n);
+    return !(worst <= kScreenThreshold && big <= (kMode == kCodeS4 ? 7.25f : 127.25f) && n == n);
 }
 
 // Exact route for the same 8 channels: two correctly rounded divisions per element.  s8 / rs8 point
 // at the channels' s and RN(1/s) in global memory.
-template <bool kFast, bool kAsym = false>
+template <bool kFast, int kMode = kCodeS8>
 __device__ __noinline__ void quantize8_exact(uint32_t x0, uint32_t x1, uint32_t x2, uint32_t x3, const float *s8,
                                              const float *rs8, float dx, float rdx, uint32_t &lo, uint32_t &hi,
                                              int z = 0)
@@ -182,9 +189,9 @@ __device__ __noinline__ void quantize8_exact(uint32_t x0, uint32_t x1, uint32_t 
         const float f = __half2float(hv);
         const float sv = __ldg(s8 + i);
         if (kFast && fabsf(f) <= 65504.0f)
-            c[i] = quantize_fast<kAsym>(f, sv, __ldg(rs8 + i), dx, rdx, z);
+            c[i] = quantize_fast<kMode>(f, sv, __ldg(rs8 + i), dx, rdx, z);
         else
-            c[i] = quantize_ieee<kAsym>(f, sv, dx, z);
+            c[i] = quantize_ieee<kMode>(f, sv, dx, z);
     }
     lo = pack4(c[0], c[1], c[2], c[3]);
     hi = pack4(c[4], c[5], c[6], c[7]);
@@ -227,7 +234,7 @@ __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_gr
 
 // The three routes for one chunk of 8 channels, cheapest first; every route that returns codes returns
 // the codes of the definition.
-template <bool kFast, bool kAsym>
+template <bool kFast, int kMode>
 __device__ __forceinline__ uint2 quantize8(const uint4 &v, const float (&c8)[8], const float *s8, const float *rs8,
                                            float dx, float rdx, int z)
 {
@@ -235,10 +242,10 @@ __device__ __forceinline__ uint2 quantize8(const uint4 &v, const float (&c8)[8],
     bool exact = true;
     if (kFast) {
         bool slow = true;
-        if (!kAsym) slow = quantize8_magic(v.x, v.y, v.z, v.w, c8, out.x, out.y);
-        exact = slow && quantize8_screen<kAsym>(v.x, v.y, v.z, v.w, c8, out.x, out.y, z);
+        if (kMode != kCodeU8) slow = quantize8_magic<kMode>(v.x, v.y, v.z, v.w, c8, out.x, out.y);
+        exact = slow && quantize8_screen<kMode>(v.x, v.y, v.z, v.w, c8, out.x, out.y, z);
     }
-    if (exact) quantize8_exact<kFast, kAsym>(v.x, v.y, v.z, v.w, s8, rs8, dx, rdx, out.x, out.y, z);
+    if (exact) quantize8_exact<kFast, kMode>(v.x, v.y, v.z, v.w, s8, rs8, dx, rdx, out.x, out.y, z);
     return out;
 }
 
@@ -254,7 +261,7 @@ __device__ __forceinline__ uint2 quantize8(const uint4 &v, const float (&c8)[8],
 // slots, kQuantRingDepth images ahead.  A thread reads back only the slots it filled itself, so no
 // barrier is involved: cp.async.wait_group orders the thread's own copies.  Loads in flight hold no
 // registers, and their number does not depend on how far the arithmetic of the current chunk has got.
-template <bool kFast, bool kAsym = false>
+template <bool kFast, int kMode = kCodeS8>
 __global__ void __launch_bounds__(256, kQuantCtasPerSm) ptq_quantize_vec8_kernel(QuantParams p)
 {
     constexpr int D = kQuantRingDepth;
@@ -269,7 +276,7 @@ __global__ void __launch_bounds__(256, kQuantCtasPerSm) ptq_quantize_vec8_kernel
     const int S = p.imgs_per_iter;
 
     const float2 d = __ldg(p.dx2 + t);
-    const int z = kAsym ? __ldg(p.zp + t) : 0;
+    const int z = kMode == kCodeU8 ? __ldg(p.zp + t) : 0;
     const float *s8 = p.s + kc * 8;          // read only on the exact route
     const float *rs8 = p.rs + kc * 8;
     float c8[8];
@@ -296,7 +303,7 @@ __global__ void __launch_bounds__(256, kQuantCtasPerSm) ptq_quantize_vec8_kernel
     while (b < p.B) {
         cp_async_wait<D - 1>();                                   // the oldest group, i.e. this slot, has landed
         const uint4 v = ring[slot][threadIdx.x];
-        *reinterpret_cast<uint2 *>(qp) = quantize8<kFast, kAsym>(v, c8, s8, rs8, d.x, d.y, z);
+        *reinterpret_cast<uint2 *>(qp) = quantize8<kFast, kMode>(v, c8, s8, rs8, d.x, d.y, z);
         // refill the slot just consumed (its value has been used above) with the image D*S further on
         if (b + D * S < p.B) cp_async_16(&ring[slot][threadIdx.x], xp + D * x_step);
         cp_async_commit();
@@ -309,7 +316,7 @@ __global__ void __launch_bounds__(256, kQuantCtasPerSm) ptq_quantize_vec8_kernel
 }
 
 // Generic path: any K, any alignment; one element per thread per step.
-template <bool kFast, bool kAsym = false>
+template <bool kFast, int kMode = kCodeS8>
 __global__ void __launch_bounds__(256) ptq_quantize_scalar_kernel(QuantParams p)
 {
     const long long total = p.M * p.K;
@@ -321,13 +328,32 @@ __global__ void __launch_bounds__(256) ptq_quantize_scalar_kernel(QuantParams p)
         const __half h = p.x[i];
         const float xf = __half2float(h);
         const unsigned short bits = __half_as_ushort(h);
-        const int z = kAsym ? __ldg(p.zp + t) : 0;
+        const int z = kMode == kCodeU8 ? __ldg(p.zp + t) : 0;
         int c;
         if (kFast && (bits & 0x7c00u) != 0x7c00u)
-            c = quantize_fast<kAsym>(xf, __ldg(p.s + k), __ldg(p.rs + k), __ldg(p.dx + t), __ldg(p.rdx + t), z);
+            c = quantize_fast<kMode>(xf, __ldg(p.s + k), __ldg(p.rs + k), __ldg(p.dx + t), __ldg(p.rdx + t), z);
         else
-            c = quantize_ieee<kAsym>(xf, __ldg(p.s + k), __ldg(p.dx + t), z);
+            c = quantize_ieee<kMode>(xf, __ldg(p.s + k), __ldg(p.dx + t), z);
         p.q[m * p.q_pitch + k] = static_cast<int8_t>(c);
+    }
+}
+
+// Two adjacent 4-bit codes (held one per byte, row pitch `pitch`) into one byte, low nibble = even
+// channel (the packing step of Appendix B.1): out[m, i] = (q[m, 2i+1] << 4) | (q[m, 2i] & 15); an odd K
+// ends the row with a zero high nibble.
+__global__ void __launch_bounds__(256) ptq_pack_int4_kernel(const int8_t *q, long long M, int K, int pitch,
+                                                            uint8_t *out)
+{
+    const int pb = (K + 1) >> 1;
+    const long long total = M * pb;
+    const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+    for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < total; i += stride) {
+        const long long m = i / pb;
+        const int j = static_cast<int>(i - m * pb);
+        const int8_t *row = q + m * pitch;
+        const int lo = row[2 * j];
+        const int hi = (2 * j + 1 < K) ? row[2 * j + 1] : 0;
+        out[i] = static_cast<uint8_t>(((hi << 4) | (lo & 15)) & 0xff);
     }
 }
 
