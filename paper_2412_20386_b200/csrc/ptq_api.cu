@@ -13,6 +13,7 @@
 #include <cstring>
 #include <mutex>
 #include <new>
+#include <utility>
 #include <vector>
 
 #include "ptq_calibrate.cuh"
@@ -188,6 +189,25 @@ int query_max_pairs()
     return cached;
 }
 
+// Launch with the programmatic-stream-serialization attribute: the kernel may begin (its set-up, up to
+// its griddep_wait()) while the previous kernel in the stream drains.  Every kernel launched this way
+// calls griddep_wait() before touching anything another kernel may have written.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kern)(KArgs...), int grid, int block, size_t smem, cudaStream_t stream, Args &&...args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(grid), 1, 1);
+    cfg.blockDim = dim3(static_cast<unsigned>(block), 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
+}
+
 // Q1 launch: codes to `q` with `q_pitch` bytes between rows.
 ptq_status_t launch_quantize(const ptq_linear *h, const void *x, long long M, void *q, int q_pitch,
                              cudaStream_t stream)
@@ -229,18 +249,18 @@ ptq_status_t launch_quantize(const ptq_linear *h, const void *x, long long M, vo
         const int grid = static_cast<int>(S * cpi / 256);
         if (h->act_bits == 4) {
             if (h->fast_div)
-                ptq::ptq_quantize_vec8_kernel<true, ptq::kCodeS4><<<grid, 256, 0, stream>>>(p);
+                PTQ_CUDA(launch_pdl(ptq::ptq_quantize_vec8_kernel<true, ptq::kCodeS4>, grid, 256, 0, stream, p));
             else
-                ptq::ptq_quantize_vec8_kernel<false, ptq::kCodeS4><<<grid, 256, 0, stream>>>(p);
+                PTQ_CUDA(launch_pdl(ptq::ptq_quantize_vec8_kernel<false, ptq::kCodeS4>, grid, 256, 0, stream, p));
         } else if (h->asym) {
             if (h->fast_div)
-                ptq::ptq_quantize_vec8_kernel<true, ptq::kCodeU8><<<grid, 256, 0, stream>>>(p);
+                PTQ_CUDA(launch_pdl(ptq::ptq_quantize_vec8_kernel<true, ptq::kCodeU8>, grid, 256, 0, stream, p));
             else
-                ptq::ptq_quantize_vec8_kernel<false, ptq::kCodeU8><<<grid, 256, 0, stream>>>(p);
+                PTQ_CUDA(launch_pdl(ptq::ptq_quantize_vec8_kernel<false, ptq::kCodeU8>, grid, 256, 0, stream, p));
         } else if (h->fast_div)
-            ptq::ptq_quantize_vec8_kernel<true><<<grid, 256, 0, stream>>>(p);
+            PTQ_CUDA(launch_pdl(ptq::ptq_quantize_vec8_kernel<true>, grid, 256, 0, stream, p));
         else
-            ptq::ptq_quantize_vec8_kernel<false><<<grid, 256, 0, stream>>>(p);
+            PTQ_CUDA(launch_pdl(ptq::ptq_quantize_vec8_kernel<false>, grid, 256, 0, stream, p));
     } else {
         long long want = (M * h->K + 255) / 256;
         const long long cap = static_cast<long long>(h->num_sms) * 8;
@@ -249,18 +269,18 @@ ptq_status_t launch_quantize(const ptq_linear *h, const void *x, long long M, vo
         const int g = static_cast<int>(want);
         if (h->act_bits == 4) {
             if (h->fast_div)
-                ptq::ptq_quantize_scalar_kernel<true, ptq::kCodeS4><<<g, 256, 0, stream>>>(p);
+                PTQ_CUDA(launch_pdl(ptq::ptq_quantize_scalar_kernel<true, ptq::kCodeS4>, g, 256, 0, stream, p));
             else
-                ptq::ptq_quantize_scalar_kernel<false, ptq::kCodeS4><<<g, 256, 0, stream>>>(p);
+                PTQ_CUDA(launch_pdl(ptq::ptq_quantize_scalar_kernel<false, ptq::kCodeS4>, g, 256, 0, stream, p));
         } else if (h->asym) {
             if (h->fast_div)
-                ptq::ptq_quantize_scalar_kernel<true, ptq::kCodeU8><<<g, 256, 0, stream>>>(p);
+                PTQ_CUDA(launch_pdl(ptq::ptq_quantize_scalar_kernel<true, ptq::kCodeU8>, g, 256, 0, stream, p));
             else
-                ptq::ptq_quantize_scalar_kernel<false, ptq::kCodeU8><<<g, 256, 0, stream>>>(p);
+                PTQ_CUDA(launch_pdl(ptq::ptq_quantize_scalar_kernel<false, ptq::kCodeU8>, g, 256, 0, stream, p));
         } else if (h->fast_div)
-            ptq::ptq_quantize_scalar_kernel<true><<<g, 256, 0, stream>>>(p);
+            PTQ_CUDA(launch_pdl(ptq::ptq_quantize_scalar_kernel<true>, g, 256, 0, stream, p));
         else
-            ptq::ptq_quantize_scalar_kernel<false><<<g, 256, 0, stream>>>(p);
+            PTQ_CUDA(launch_pdl(ptq::ptq_quantize_scalar_kernel<false>, g, 256, 0, stream, p));
     }
     g_launches.fetch_add(1, std::memory_order_relaxed);
     PTQ_CUDA(cudaGetLastError());
@@ -288,11 +308,11 @@ ptq_status_t launch_quantize_dynamic(const ptq_linear *h, const void *x, long lo
     if (want > cap) want = cap;
     if (want < 1) want = 1;
     if (!vec)
-        ptq::ptq_quantize_dynamic_scalar_kernel<<<static_cast<int>(want), 256, 0, stream>>>(p);
+        PTQ_CUDA(launch_pdl(ptq::ptq_quantize_dynamic_scalar_kernel, static_cast<int>(want), 256, 0, stream, p));
     else if (h->fast_div)
-        ptq::ptq_quantize_dynamic_vec8_kernel<true><<<static_cast<int>(want), 256, 0, stream>>>(p);
+        PTQ_CUDA(launch_pdl(ptq::ptq_quantize_dynamic_vec8_kernel<true>, static_cast<int>(want), 256, 0, stream, p));
     else
-        ptq::ptq_quantize_dynamic_vec8_kernel<false><<<static_cast<int>(want), 256, 0, stream>>>(p);
+        PTQ_CUDA(launch_pdl(ptq::ptq_quantize_dynamic_vec8_kernel<false>, static_cast<int>(want), 256, 0, stream, p));
     g_launches.fetch_add(1, std::memory_order_relaxed);
     PTQ_CUDA(cudaGetLastError());
     return PTQ_OK;
@@ -375,9 +395,9 @@ ptq_status_t launch_gemm(const ptq_linear *h, const void *codes, long long M, vo
     const long long tiles = static_cast<long long>(p.m_tiles) * p.n_tiles;
     const int grid = static_cast<int>(tiles < h->num_sms ? tiles : h->num_sms);
     if (acc_out)
-        ptq::ptq_gemm_dequant_kernel<true><<<grid, ptq::kGemmThreads, ptq::kGemmSmemBytes, stream>>>(tmA, h->tmW, tmY, p);
+        PTQ_CUDA(launch_pdl(ptq::ptq_gemm_dequant_kernel<true>, grid, ptq::kGemmThreads, ptq::kGemmSmemBytes, stream, tmA, h->tmW, tmY, p));
     else
-        ptq::ptq_gemm_dequant_kernel<false><<<grid, ptq::kGemmThreads, ptq::kGemmSmemBytes, stream>>>(tmA, h->tmW, tmY, p);
+        PTQ_CUDA(launch_pdl(ptq::ptq_gemm_dequant_kernel<false>, grid, ptq::kGemmThreads, ptq::kGemmSmemBytes, stream, tmA, h->tmW, tmY, p));
     g_launches.fetch_add(1, std::memory_order_relaxed);
     PTQ_CUDA(cudaGetLastError());
     return PTQ_OK;

@@ -271,6 +271,11 @@ ptq_gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_holder;
 
+    // The set-up above touched nothing another kernel writes.  From here on the codes (and, for the
+    // dynamic comparator, the row steps) of the quantize kernel launched just before are read.
+    griddep_wait();
+    griddep_launch_dependents();
+
     const int total_tiles = p.m_tiles * p.n_tiles;
 
     if (warp == 0) {

@@ -10,6 +10,8 @@
 #include <cuda_fp16.h>
 #include <stdint.h>
 
+#include "ptx_sm100.cuh"
+
 namespace ptq {
 
 // a / d, correctly rounded (binary32, round-to-nearest-even), given r = RN(1/d).
@@ -293,6 +295,10 @@ __global__ void __launch_bounds__(256, kQuantCtasPerSm) ptq_quantize_vec8_kernel
     int8_t *qp = p.q + b * q_img + static_cast<long long>(t) * p.q_pitch + kc * 8;
     const long long x_step = S * x_img, q_step = S * q_img;
 
+    // Everything above read only the layer's own parameters; x may come from the kernel before this one.
+    griddep_wait();
+    griddep_launch_dependents();
+
     // fill the ring: slot i holds image b + i*S (one commit group per slot, empty past the last image)
 #pragma unroll
     for (int i = 0; i < D; ++i) {
@@ -319,6 +325,8 @@ __global__ void __launch_bounds__(256, kQuantCtasPerSm) ptq_quantize_vec8_kernel
 template <bool kFast, int kMode = kCodeS8>
 __global__ void __launch_bounds__(256) ptq_quantize_scalar_kernel(QuantParams p)
 {
+    griddep_wait();
+    griddep_launch_dependents();
     const long long total = p.M * p.K;
     const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
     for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < total; i += stride) {

@@ -80,6 +80,8 @@ __global__ void __launch_bounds__(256, PTQ_DYN_CTAS_PER_SM) ptq_quantize_dynamic
     const int cpr = p.K >> 3;
     const float4 *s4 = reinterpret_cast<const float4 *>(p.s);
     const float4 *r4 = reinterpret_cast<const float4 *>(p.rs);
+    griddep_wait();
+    griddep_launch_dependents();
 
     for (long long m0 = warp * R; m0 < p.M; m0 += nwarps * R) {
         const int rows = static_cast<int>(p.M - m0 < R ? p.M - m0 : R);
@@ -158,6 +160,8 @@ __global__ void __launch_bounds__(256, PTQ_DYN_CTAS_PER_SM) ptq_quantize_dynamic
 // Generic path: any K and alignment; one warp per row, one element per lane and step, IEEE divisions.
 __global__ void __launch_bounds__(256) ptq_quantize_dynamic_scalar_kernel(DynQuantParams p)
 {
+    griddep_wait();
+    griddep_launch_dependents();
     const int lane = threadIdx.x & 31;
     const long long warp = static_cast<long long>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const long long nwarps = static_cast<long long>(gridDim.x) * (blockDim.x >> 5);

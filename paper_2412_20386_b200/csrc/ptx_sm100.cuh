@@ -32,6 +32,14 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
 
+// Programmatic dependent launch (sm_90+).  A kernel launched with the programmatic-stream-serialization
+// attribute may start while its predecessor in the stream is still running; griddep_wait() blocks the
+// calling thread until every prerequisite grid has completed and its memory operations are visible
+// (a no-op when the launch carried no such dependency).  griddep_launch_dependents() lets the NEXT
+// kernel's CTAs be scheduled as soon as resources free up instead of at this grid's very end.
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ void fence_mbar_init()
 {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
