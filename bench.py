@@ -504,10 +504,10 @@ def run_ours(args, specs, rank, world, local_rank):
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised
 # under profiles/; keyed by (kernel, workload, layer).  An entry is removed when its kernel changes.
 TRAFFIC = {
-    ("ptq_gemm_dequant_kernel", "c3", "in_proj"): 41.175296e6 + 255.838976e6,
-    ("ptq_gemm_dequant_kernel", "c3", "out_proj"): 78.698240e6 + 34.846976e6,
-    ("ptq_quantize_kernel", "c3", "in_proj"): 77.514752e6 + 10.142720e6,
-    ("ptq_quantize_kernel", "c3", "out_proj"): 155.153664e6 + 47.354624e6,
+    ("ptq_gemm_dequant_kernel", "c3", "in_proj"): 41.221120e6 + 256.052480e6,
+    ("ptq_gemm_dequant_kernel", "c3", "out_proj"): 78.699776e6 + 34.394112e6,
+    ("ptq_quantize_kernel", "c3", "in_proj"): 77.508096e6 + 10.753792e6,
+    ("ptq_quantize_kernel", "c3", "out_proj"): 155.139072e6 + 47.510784e6,
 }
 
 
