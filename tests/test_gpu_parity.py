@@ -180,6 +180,22 @@ def test_odd_shapes_and_ragged_tiles(env, K, N, T, B):
     check_layer(ptq, torch, spec, full=True)
 
 
+def test_seeded_random_shapes(env):
+    """Sixteen seeded random (K, N, T, B): every kernel variant the shape and alignment select, every flag."""
+    ptq, torch = env
+    rng = np.random.default_rng(20241228)
+    for i in range(16):
+        K = int(rng.integers(1, 700))
+        N = int(rng.integers(1, 600))
+        T = int(rng.integers(1, 60))
+        B = int(rng.integers(1, 12)) * int(rng.choice([1, 1, 7]))
+        if i % 4 == 0:
+            K = (K + 7) // 8 * 8                     # some shapes on the vector paths
+            N = (N + 7) // 8 * 8
+        spec = wl.LinearSpec(8, i, i % 4, "rand%d" % i, B, T, K, N, bias=bool(i & 1))
+        check_layer(ptq, torch, spec, full=True)
+
+
 def test_fused_flag_is_reported_and_needs_no_workspace(env):
     ptq, torch = env
     for spec, want in ((CFG[3][0], True), (CFG[3][1], True), (CFG[1][2], False),
