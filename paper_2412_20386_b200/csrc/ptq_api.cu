@@ -337,10 +337,13 @@ ptq_status_t launch_gemm(const ptq_linear *h, const void *codes, long long M, vo
                                   ptq::kBK, ptq::kBM);
     if (st != PTQ_OK) return st;
     const bool tma_store = (h->N % 8 == 0) && (reinterpret_cast<uintptr_t>(y) % 16 == 0);
+    const int m_tiles_ = static_cast<int>((M + ptq::kBM - 1) / ptq::kBM);
+    const bool use_pair = want_pair && h->max_pairs > 0 &&
+                          static_cast<long long>((m_tiles_ + 1) / 2) * h->n_tiles >= h->max_pairs;
     if (tma_store) {
         st = make_map_2d(&tmY, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, y, static_cast<unsigned long long>(h->N),
                          static_cast<unsigned long long>(M), static_cast<unsigned long long>(h->N) * 2,
-                         ptq::kStoreBoxCols, 32);
+                         use_pair ? ptq::kStoreBoxCols : ptq::kStreamBoxCols, 32);
         if (st != PTQ_OK) return st;
     } else {
         tmY = h->tmW;   // never dereferenced by the kernel in this mode
@@ -368,8 +371,7 @@ ptq_status_t launch_gemm(const ptq_linear *h, const void *codes, long long M, vo
     p.zp = h->d_zp;
     p.wsum = h->d_wsum;
 
-    const long long pair_tiles = static_cast<long long>((p.m_tiles + 1) / 2) * p.n_tiles;
-    if (want_pair && h->max_pairs > 0 && pair_tiles >= h->max_pairs) {
+    if (use_pair) {
         // enough 256-row tiles to occupy every CTA pair: cta_group::2 kernel (half the weight bytes per CTA)
         const int npairs = h->max_pairs;
         cudaLaunchConfig_t cfg = {};

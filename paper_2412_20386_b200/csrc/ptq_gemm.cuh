@@ -13,8 +13,8 @@
 //   warp 1      owns TMEM (512 columns = two 128 x 256 accumulators) and issues the MMAs; a
 //               tcgen05.commit frees each shared-memory stage and publishes each accumulator
 //   warps 2..9  epilogue: tcgen05.ld (lane quarter = warp % 4; the two warps of a quarter take
-//               alternate 64-column steps), scale, convert, stage 32 x 32 fp16 boxes in swizzled shared
-//               memory (two per warp) and write them with TMA stores
+//               alternate 64-column steps), scale, convert, stage each step as one 32 x 64 fp16 box in
+//               swizzled shared memory (128-byte rows) and write it with one TMA store
 // While the epilogue drains accumulator i the MMA warp already fills accumulator i^1.
 #pragma once
 
@@ -40,8 +40,17 @@ constexpr int kStagingBytesPerWarp = 2 * kStoreBoxBytes;  // two boxes: one bein
 constexpr int kGemmThreads = 32 * (2 + kNumEpiWarps);
 constexpr int kTmemCols = 512;
 constexpr int kNumBarriers = 2 * kStages + 4;
+// The streaming kernel stages one 32-row x 64-column box per warp (128-byte rows, 128-byte swizzle)
+// and stores a whole 64-column step with one TMA store; the pair and fused kernels use the two
+// 32-column boxes above.
+#ifndef PTQ_STORE_BOX64
+#define PTQ_STORE_BOX64 1
+#endif
+constexpr bool kStreamBox64 = PTQ_STORE_BOX64 != 0;
+constexpr int kStreamBoxCols = kStreamBox64 ? 64 : kStoreBoxCols;
+constexpr int kStreamStagingPerWarp = kStreamBox64 ? 32 * 128 : kStagingBytesPerWarp;
 constexpr int kGemmSmemBytes =
-    1024 + kStages * kStageBytes + kNumEpiWarps * kStagingBytesPerWarp + kNumBarriers * 8 + 16;
+    1024 + kStages * kStageBytes + kNumEpiWarps * kStreamStagingPerWarp + kNumBarriers * 8 + 16;
 
 struct GemmParams {
     long long M;
@@ -108,6 +117,27 @@ __device__ __forceinline__ void convert_stage32(const uint32_t (&v)[32], float d
     }
 }
 
+// Same for one half (32 columns) of a 128-byte row of a 64-column box: chunks 4*half .. 4*half+3, chunk
+// index XOR (row & 7): the 128-byte swizzle.
+__device__ __forceinline__ void convert_stage32_sw128(const uint32_t (&v)[32], float dxr, const float *dw,
+                                                      const float *bias, uint32_t row_addr, int lane, int half)
+{
+    const uint32_t sw = static_cast<uint32_t>(lane & 7);
+#pragma unroll
+    for (int jj = 0; jj < 4; ++jj) {
+        const float4 w0 = __ldg(reinterpret_cast<const float4 *>(dw + 8 * jj));
+        const float4 w1 = __ldg(reinterpret_cast<const float4 *>(dw + 8 * jj + 4));
+        const float4 b0 = __ldg(reinterpret_cast<const float4 *>(bias + 8 * jj));
+        const float4 b1 = __ldg(reinterpret_cast<const float4 *>(bias + 8 * jj + 4));
+        uint4 o;
+        o.x = pack_half2(dequant_one(v[8 * jj + 0], dxr, w0.x, b0.x), dequant_one(v[8 * jj + 1], dxr, w0.y, b0.y));
+        o.y = pack_half2(dequant_one(v[8 * jj + 2], dxr, w0.z, b0.z), dequant_one(v[8 * jj + 3], dxr, w0.w, b0.w));
+        o.z = pack_half2(dequant_one(v[8 * jj + 4], dxr, w1.x, b1.x), dequant_one(v[8 * jj + 5], dxr, w1.y, b1.y));
+        o.w = pack_half2(dequant_one(v[8 * jj + 6], dxr, w1.z, b1.z), dequant_one(v[8 * jj + 7], dxr, w1.w, b1.w));
+        st_shared_v4(row_addr + ((static_cast<uint32_t>(4 * half + jj) ^ sw) << 4), o);
+    }
+}
+
 // Plain masked stores of 32 columns of this thread's row (any N, any alignment of y).
 __device__ __forceinline__ void convert_store32_plain(const uint32_t (&v)[32], float dxr, const float *dw,
                                                       const float *bias, __half *yrow, int n_first, int N,
@@ -164,7 +194,7 @@ __device__ __forceinline__ void store_acc32(const uint32_t (&v)[32], int32_t *ar
 // is not on the warp's critical path.  Returns the updated count of staged boxes.
 // kLowReg = false keeps both TMEM loads of a step in flight (64 accumulator registers);
 // kLowReg = true loads 32 columns at a time (for kernels whose thread count caps the registers).
-template <bool kDebugAcc, bool kLowReg = false>
+template <bool kDebugAcc, bool kLowReg = false, bool kBox64 = false>
 __device__ __forceinline__ uint32_t epilogue_tile(const GemmParams &p, const CUtensorMap *tmY, uint32_t tmem_row,
                                                   long long m_row0, int n0, float dxr, uint32_t staging,
                                                   uint32_t nboxes, int lane, int col_half, int zr = 0)
@@ -199,7 +229,26 @@ __device__ __forceinline__ uint32_t epilogue_tile(const GemmParams &p, const CUt
             if (kDebugAcc) {
                 if (p.acc_out != nullptr && row_ok) store_acc32(v, p.acc_out + m * p.N, n_half, p.N);
             }
-            if (p.use_tma_store) {
+            if (kBox64 && p.use_tma_store) {
+                // one 64-column box per step: wait until the previous step's store has read the box, fill
+                // its two halves, store once
+                if (half == 0) {
+                    if (nboxes >= 1u && lane == 0) bulk_wait_group_read<0>();
+                    __syncwarp();
+                }
+                convert_stage32_sw128(v, dxr, p.dw + n_half, p.bias + n_half, staging + static_cast<uint32_t>(lane) * 128u,
+                                      lane, half);
+                if (half == 1) {
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        if (n_first < p.N && m_row0 < p.M)
+                            tma_store_2d(tmY, n_first, static_cast<int>(m_row0), staging);   // clipped at N and M
+                        bulk_commit_group();
+                    }
+                    ++nboxes;
+                }
+            } else if (p.use_tma_store) {
                 const uint32_t box = staging + (nboxes & 1u) * kStoreBoxBytes;
                 if (nboxes >= 2u && lane == 0) bulk_wait_group_read<1>();   // the store that last used this box has read it
                 __syncwarp();
@@ -235,7 +284,7 @@ ptq_gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     const uint32_t base = (raw + 1023u) & ~1023u;                    // swizzled tiles need 1024-byte alignment
     uint8_t *base_ptr = smem_raw + (base - raw);
     const uint32_t staging_base = base + kStages * kStageBytes;
-    const uint32_t bar_off = kStages * kStageBytes + kNumEpiWarps * kStagingBytesPerWarp;
+    const uint32_t bar_off = kStages * kStageBytes + kNumEpiWarps * kStreamStagingPerWarp;
     const uint32_t bar_base = base + bar_off;
     auto full_bar = [&](uint32_t s) { return bar_base + 8u * s; };
     auto empty_bar = [&](uint32_t s) { return bar_base + 8u * (kStages + s); };
@@ -351,7 +400,7 @@ ptq_gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         // ------------------------------------------------------------------ epilogue warps
         const int quarter = warp & 3;                // TMEM lanes [32*quarter, 32*quarter+32)
         const int col_half = (warp - 2) >> 2;        // which of the alternating 64-column boxes
-        const uint32_t staging = staging_base + static_cast<uint32_t>(warp - 2) * kStagingBytesPerWarp;
+        const uint32_t staging = staging_base + static_cast<uint32_t>(warp - 2) * kStreamStagingPerWarp;
         uint32_t buf = 0, bphase = 0, nboxes = 0;
         for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
             const int m_tile = tile / p.n_tiles;
@@ -366,8 +415,8 @@ ptq_gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             if (!got) break;
             tc_fence_after_sync();
             const uint32_t tmem_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * kMaxBN;
-            nboxes = epilogue_tile<kDebugAcc>(p, &tmY, tmem_row, m_row0, n_tile * p.BN, dxr, staging, nboxes, lane, col_half,
-                                              zr);
+            nboxes = epilogue_tile<kDebugAcc, false, kStreamBox64>(p, &tmY, tmem_row, m_row0, n_tile * p.BN, dxr, staging,
+                                                                   nboxes, lane, col_half, zr);
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(tempty_bar(buf));
