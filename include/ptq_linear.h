@@ -29,6 +29,10 @@
  *     so concurrent forwards on different streams are allowed as long as they
  *     use different workspaces (each handle also carries one device status
  *     word that all its launches may set; see ptq_linear_device_status).
+ *   - The quantize and GEMM kernels are launched with the programmatic-stream-serialization
+ *     attribute: their set-up may run while the previous kernel on the stream drains, and each waits
+ *     for that kernel's completion before it reads or writes any buffer.  Results and ordering are
+ *     those of plain stream order.
  *   - Requires a device of compute capability 10.0 (sm_100a); create fails
  *     with PTQ_ERR_ARCH elsewhere.  There is no CPU or generic-GPU fallback.
  */
@@ -58,7 +62,8 @@ typedef enum {
 
 /* Flags for create / forward. */
 #define PTQ_FLAG_NONE            0u
-#define PTQ_FLAG_FUSED_PROLOGUE  1u   /* F1: quantize inside the GEMM kernel; no int8 round trip, no workspace */
+#define PTQ_FLAG_FUSED_PROLOGUE  1u   /* F1: quantize inside the GEMM kernel; no int8 round trip, no workspace
+                                         (same bits; at present slower than the two-kernel path) */
 #define PTQ_FLAG_CTA_PAIR        2u   /* two-kernel path: run G1+E1 on CTA pairs (tcgen05 cta_group::2, 256-row tiles,
                                          half the weight bytes per CTA) when the batch has enough rows; same results */
 
