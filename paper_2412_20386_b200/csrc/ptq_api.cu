@@ -343,7 +343,7 @@ ptq_status_t launch_gemm(const ptq_linear *h, const void *codes, long long M, vo
     if (tma_store) {
         st = make_map_2d(&tmY, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, y, static_cast<unsigned long long>(h->N),
                          static_cast<unsigned long long>(M), static_cast<unsigned long long>(h->N) * 2,
-                         use_pair ? ptq::kStoreBoxCols : ptq::kStreamBoxCols, 32);
+                         ptq::kStreamBoxCols, 32);
         if (st != PTQ_OK) return st;
     } else {
         tmY = h->tmW;   // never dereferenced by the kernel in this mode

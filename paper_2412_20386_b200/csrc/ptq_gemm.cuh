@@ -40,9 +40,9 @@ constexpr int kStagingBytesPerWarp = 2 * kStoreBoxBytes;  // two boxes: one bein
 constexpr int kGemmThreads = 32 * (2 + kNumEpiWarps);
 constexpr int kTmemCols = 512;
 constexpr int kNumBarriers = 2 * kStages + 4;
-// The streaming kernel stages one 32-row x 64-column box per warp (128-byte rows, 128-byte swizzle)
-// and stores a whole 64-column step with one TMA store; the pair and fused kernels use the two
-// 32-column boxes above.
+// The streaming and CTA-pair kernels stage one 32-row x 64-column box per warp (128-byte rows, 128-byte
+// swizzle) and store a whole 64-column step with one TMA store; the fused kernel uses the two 32-column
+// boxes above.
 #ifndef PTQ_STORE_BOX64
 #define PTQ_STORE_BOX64 1
 #endif
@@ -599,8 +599,8 @@ ptq_gemm_dequant_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __gr
             if (!got) break;
             tc_fence_after_sync();
             const uint32_t tmem_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * kMaxBN;
-            nboxes = epilogue_tile<kDebugAcc>(p, &tmY, tmem_row, m_row0, n_tile * p.BN, dxr, staging, nboxes, lane,
-                                              col_half);
+            nboxes = epilogue_tile<kDebugAcc, false, kStreamBox64>(p, &tmY, tmem_row, m_row0, n_tile * p.BN, dxr, staging,
+                                                                   nboxes, lane, col_half);
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive_remote(tempty_bar(buf), 0u);     // the leader's MMA thread waits on it
