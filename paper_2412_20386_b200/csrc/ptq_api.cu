@@ -123,7 +123,7 @@ struct ptq_linear {
     CUtensorMap tmW;
     CUtensorMap tmWh;          // same weights, box of BN/2 rows: the half tile one CTA of a pair loads
     int max_pairs = 0;         // resident 2-CTA clusters of the pair kernel on this device (0: not available)
-    // A-stationary kernel (fused, and the two-kernel path's GEMM when the code panel fits shared memory)
+    // tiling of the fused (A-stationary) kernel
     bool as_ok = false;
     int as_BN = 0, as_n_tiles = 0, as_w_stages = 0, as_w_stage_bytes = 0, as_staging = 0, as_smem = 0;
     CUtensorMap tmWas;
@@ -434,31 +434,21 @@ void choose_astat(ptq_linear *h)
 }
 
 template <typename Kern>
-ptq_status_t launch_astat_kernel(Kern kern, int threads, const ptq_linear *h, const CUtensorMap &tmA,
-                                 const CUtensorMap &tmY, const ptq::FusedParams &fp, int grid, cudaStream_t stream)
+ptq_status_t launch_fused_kernel(Kern kern, const ptq_linear *h, const CUtensorMap &tmY, const ptq::FusedParams &fp,
+                                 int grid, cudaStream_t stream)
 {
     PTQ_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ptq::kFusedSmemLimit));
-    kern<<<grid, threads, h->as_smem, stream>>>(tmA, h->tmWas, tmY, fp);
+    kern<<<grid, ptq::kFusedThreadsQuant, h->as_smem, stream>>>(h->tmWas, tmY, fp);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     PTQ_CUDA(cudaGetLastError());
     return PTQ_OK;
 }
 
-// A-stationary launch.  quantize = true: `src` is x fp16 [M,K] (Q1 + G1 + E1 in one kernel);
-// quantize = false: `src` is the code matrix [M,Kpad] (G1 + E1).
-ptq_status_t launch_astat(const ptq_linear *h, const void *src, bool quantize, long long M, void *y, void *acc_out,
-                          cudaStream_t stream)
+// F1 launch: x fp16 [M,K] -> y (Q1 + G1 + E1 in one kernel, the code panel of a row tile resident in shared memory).
+ptq_status_t launch_fused(const ptq_linear *h, const void *x, long long M, void *y, void *acc_out, cudaStream_t stream)
 {
-    CUtensorMap tmA, tmY;
+    CUtensorMap tmY;
     ptq_status_t st;
-    if (!quantize) {
-        st = make_map_2d(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, src, static_cast<unsigned long long>(h->K),
-                         static_cast<unsigned long long>(M), static_cast<unsigned long long>(h->Kpad), ptq::kBK,
-                         ptq::kBM);
-        if (st != PTQ_OK) return st;
-    } else {
-        tmA = h->tmWas;   // unused by the kernel in this mode
-    }
     const bool aligned = (h->N % 8 == 0) && (reinterpret_cast<uintptr_t>(y) % 16 == 0);
     const bool tma_store = aligned && h->as_staging;
     if (tma_store) {
@@ -467,7 +457,7 @@ ptq_status_t launch_astat(const ptq_linear *h, const void *src, bool quantize, l
                          ptq::kStoreBoxCols, 32);
         if (st != PTQ_OK) return st;
     } else {
-        tmY = h->tmWas;
+        tmY = h->tmWas;   // never dereferenced by the kernel in this mode
     }
     ptq::FusedParams fp;
     ptq::GemmParams &p = fp.g;
@@ -491,7 +481,7 @@ ptq_status_t launch_astat(const ptq_linear *h, const void *src, bool quantize, l
     p.y_vec8 = (aligned && !tma_store) ? 1 : 0;
     p.zp = nullptr;
     p.wsum = nullptr;
-    fp.x = static_cast<const __half *>(quantize ? src : nullptr);
+    fp.x = static_cast<const __half *>(x);
     fp.s = h->d_s;
     fp.rs = h->d_rs;
     fp.dx2 = h->d_dx2;
@@ -500,25 +490,11 @@ ptq_status_t launch_astat(const ptq_linear *h, const void *src, bool quantize, l
     fp.has_staging = h->as_staging;
     const int grid = p.m_tiles < h->num_sms ? p.m_tiles : h->num_sms;
     const bool dbg = acc_out != nullptr;
-    if (quantize) {
-        const int th = ptq::kFusedThreadsQuant;
-        if (h->fast_div)
-            return dbg ? launch_astat_kernel(ptq::ptq_fused_linear_kernel<true, true, true>, th, h, tmA, tmY, fp, grid, stream)
-                       : launch_astat_kernel(ptq::ptq_fused_linear_kernel<true, true, false>, th, h, tmA, tmY, fp, grid, stream);
-        return dbg ? launch_astat_kernel(ptq::ptq_fused_linear_kernel<true, false, true>, th, h, tmA, tmY, fp, grid, stream)
-                   : launch_astat_kernel(ptq::ptq_fused_linear_kernel<true, false, false>, th, h, tmA, tmY, fp, grid, stream);
-    }
-    const int th = ptq::kFusedThreadsPlain;
-    return dbg ? launch_astat_kernel(ptq::ptq_fused_linear_kernel<false, true, true>, th, h, tmA, tmY, fp, grid, stream)
-               : launch_astat_kernel(ptq::ptq_fused_linear_kernel<false, true, false>, th, h, tmA, tmY, fp, grid, stream);
-}
-
-// G1 + E1 on codes.  The streaming kernels keep more bytes in flight from L2 than the A-stationary one
-// (whose resident code panel leaves little shared memory for weight stages) and measure faster.
-ptq_status_t launch_gemm_any(const ptq_linear *h, const void *codes, long long M, void *y, void *acc_out,
-                             cudaStream_t stream, bool want_pair = false)
-{
-    return launch_gemm(h, codes, M, y, acc_out, stream, want_pair);
+    if (h->fast_div)
+        return dbg ? launch_fused_kernel(ptq::ptq_fused_linear_kernel<true, true>, h, tmY, fp, grid, stream)
+                   : launch_fused_kernel(ptq::ptq_fused_linear_kernel<true, false>, h, tmY, fp, grid, stream);
+    return dbg ? launch_fused_kernel(ptq::ptq_fused_linear_kernel<false, true>, h, tmY, fp, grid, stream)
+               : launch_fused_kernel(ptq::ptq_fused_linear_kernel<false, false>, h, tmY, fp, grid, stream);
 }
 
 bool fused_usable(const ptq_linear *h) { return h->as_ok && h->K % 16 == 0; }
@@ -800,7 +776,7 @@ ptq_status_t ptq_linear_gemm_dequant(const ptq_linear_t *h, const void *q_int8, 
     const long long M = static_cast<long long>(B) * h->T;
     if (ranges_overlap(q_int8, static_cast<size_t>(M) * h->Kpad, y_fp16, static_cast<size_t>(M) * h->N * 2))
         return fail(PTQ_ERR_VALUE, "q and y overlap");
-    return launch_gemm_any(h, q_int8, M, y_fp16, nullptr, static_cast<cudaStream_t>(stream));
+    return launch_gemm(h, q_int8, M, y_fp16, nullptr, static_cast<cudaStream_t>(stream));
 }
 
 ptq_status_t ptq_linear_forward_debug(const ptq_linear_t *h, const void *x_fp16, int B, void *y_fp16,
@@ -815,7 +791,7 @@ ptq_status_t ptq_linear_forward_debug(const ptq_linear_t *h, const void *x_fp16,
     if ((flags & PTQ_FLAG_FUSED_PROLOGUE) && fused_usable(h) && reinterpret_cast<uintptr_t>(x_fp16) % 16 == 0) {
         // F1: one kernel, no workspace.  The codes never exist in memory; a requested tap is produced by
         // the quantize kernel on its own.
-        if ((st = launch_astat(h, x_fp16, true, M, y_fp16, acc_int32_out, s)) != PTQ_OK) return st;
+        if ((st = launch_fused(h, x_fp16, M, y_fp16, acc_int32_out, s)) != PTQ_OK) return st;
         if (q_int8_out) return launch_quantize(h, x_fp16, M, q_int8_out, h->K, s);
         return PTQ_OK;
     }
@@ -828,7 +804,7 @@ ptq_status_t ptq_linear_forward_debug(const ptq_linear_t *h, const void *x_fp16,
         ranges_overlap(workspace, need, x_fp16, static_cast<size_t>(M) * h->K * 2))
         return fail(PTQ_ERR_VALUE, "workspace overlaps x or y");
     if ((st = launch_quantize(h, x_fp16, M, workspace, h->Kpad, s)) != PTQ_OK) return st;
-    if ((st = launch_gemm_any(h, workspace, M, y_fp16, acc_int32_out, s, (flags & PTQ_FLAG_CTA_PAIR) != 0)) != PTQ_OK)
+    if ((st = launch_gemm(h, workspace, M, y_fp16, acc_int32_out, s, (flags & PTQ_FLAG_CTA_PAIR) != 0)) != PTQ_OK)
         return st;
     if (q_int8_out)
         PTQ_CUDA(cudaMemcpy2DAsync(q_int8_out, h->K, workspace, h->Kpad, h->K, static_cast<size_t>(M),
@@ -858,7 +834,7 @@ ptq_status_t ptq_linear_forward_static(const ptq_linear_t *h, const void *x_fp16
     if ((st = static_scratch_address(h->device, &scratch)) != PTQ_OK) return st;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if ((st = launch_quantize(h, x_fp16, M, scratch, h->Kpad, s)) != PTQ_OK) return st;
-    return launch_gemm_any(h, scratch, M, y_fp16, nullptr, s);
+    return launch_gemm(h, scratch, M, y_fp16, nullptr, s);
 }
 
 ptq_status_t ptq_search_act_step(int K, int T, const void *xcal_fp16, int Bc, const float *smooth,

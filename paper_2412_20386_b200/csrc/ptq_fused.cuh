@@ -4,15 +4,12 @@
 //
 // A CTA owns one 128-row panel of activations at a time and keeps its int8 codes in shared memory
 // for ALL output tiles of that panel: the codes are produced once per row (not once per output
-// tile), and per output tile only the weight tile is streamed in (from L2).  Two ways to fill the
-// panel, selected at compile time:
-//   kQuantize = true   four quantizer warps load fp16 x (16-byte loads), quantize it in registers and
-//                      write the codes straight into the 128-byte-swizzled K-major layout the MMA
-//                      reads (fence.proxy.async + mbarrier arrive)
-//   kQuantize = false  the codes already exist in memory (workspace); TMA loads them
+// tile), and per output tile only the weight tile is streamed in (from L2).  Four quantizer warps
+// load fp16 x (16-byte loads), quantize it in registers and write the codes straight into the
+// 128-byte-swizzled K-major layout the MMA reads (fence.proxy.async + mbarrier arrive).
 //
-// Warps: 0 = TMA producer (weights; codes when !kQuantize), 1 = TMEM owner + MMA issuer,
-// 2..9 = epilogue (shared with the plain GEMM kernel), 10..13 = quantizers (kQuantize only).
+// Warps: 0 = TMA producer (weights), 1 = TMEM owner + MMA issuer,
+// 2..9 = epilogue (shared with the plain GEMM kernel), 10..13 = quantizers.
 // Barriers: pfull/pempty per panel k-block (filled once per panel, freed by the commit after the last
 // output tile has read it), wfull/wempty per weight stage, tfull/tempty per TMEM accumulator.
 // While the last output tile of panel i still runs, the k-blocks it has finished with are already
@@ -32,13 +29,12 @@ constexpr int kFusedMaxKBlocks = 12;                      // panel of at most 12
 constexpr int kFusedMaxWStages = 4;
 constexpr int kFusedQuantWarps = 4;
 constexpr int kFusedThreadsQuant = 32 * (2 + kNumEpiWarps + kFusedQuantWarps);   // 448
-constexpr int kFusedThreadsPlain = 32 * (2 + kNumEpiWarps);                      // 320
 constexpr int kFusedNumBarriers = 2 * kFusedMaxKBlocks + 2 * kFusedMaxWStages + 4;
 constexpr int kFusedSmemLimit = 232448;                   // 227 KB opt-in maximum per CTA
 
 struct FusedParams {
     GemmParams g;            // BN / n_tiles here are the fused kernel's own tiling
-    const __half *x;         // [M,K] fp16 (kQuantize)
+    const __half *x;         // [M,K] fp16
     const float *s;          // [K]
     const float *rs;         // [K] RN(1/s)
     const float2 *dx2;       // [T] {dx, RN(1/dx)}
@@ -53,10 +49,10 @@ __host__ __device__ inline int fused_smem_bytes(int k_blocks, int w_stages, int 
            (has_staging ? kNumEpiWarps * kStagingBytesPerWarp : 0) + kFusedNumBarriers * 8 + 16;
 }
 
-template <bool kQuantize, bool kFast, bool kDebugAcc>
-__global__ void __launch_bounds__(kQuantize ? kFusedThreadsQuant : kFusedThreadsPlain, 1)
-ptq_fused_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
-                        const __grid_constant__ CUtensorMap tmY, const FusedParams fp)
+template <bool kFast, bool kDebugAcc>
+__global__ void __launch_bounds__(kFusedThreadsQuant, 1)
+ptq_fused_linear_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmY,
+                        const FusedParams fp)
 {
     const GemmParams &p = fp.g;
     extern __shared__ uint8_t smem_raw[];
@@ -84,7 +80,7 @@ ptq_fused_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
 
     if (threadIdx.x == 0) {
         for (int kb = 0; kb < p.k_blocks; ++kb) {
-            mbar_init(pfull_bar(kb), kQuantize ? 32u * kFusedQuantWarps : 1u);
+            mbar_init(pfull_bar(kb), 32u * kFusedQuantWarps);
             mbar_init(pempty_bar(kb), 1);
         }
         for (int s = 0; s < fp.w_stages; ++s) {
@@ -98,7 +94,6 @@ ptq_fused_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         *abort_flag = 0u;
         fence_mbar_init();
         prefetch_tensormap(&tmW);
-        if (!kQuantize) prefetch_tensormap(&tmA);
         if (p.use_tma_store) prefetch_tensormap(&tmY);
     }
     if (warp == 1) {
@@ -113,22 +108,12 @@ ptq_fused_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            uint32_t stage = 0, phase = 0, it = 0;
-            uint32_t w_issued = 0, p_issued = 0;
+            uint32_t stage = 0, phase = 0;
+            uint32_t w_issued = 0;
             bool ok = true;
-            for (int m_tile = blockIdx.x; m_tile < p.m_tiles && ok; m_tile += gridDim.x, ++it) {
+            for (int m_tile = blockIdx.x; m_tile < p.m_tiles && ok; m_tile += gridDim.x) {
                 for (int n_tile = 0; n_tile < p.n_tiles && ok; ++n_tile) {
                     for (int kb = 0; kb < p.k_blocks; ++kb) {
-                        if (!kQuantize && n_tile == 0) {
-                            // codes of this panel, k-block by k-block, interleaved with the first weight tile
-                            if (!mbar_wait(pempty_bar(kb), (it & 1u) ^ 1u, abort_flag, p.status)) {
-                                ok = false;
-                                break;
-                            }
-                            mbar_arrive_expect_tx(pfull_bar(kb), kATileBytes);
-                            tma_load_2d(panel_base + kb * kATileBytes, &tmA, kb * kBK, m_tile * kBM, pfull_bar(kb));
-                            ++p_issued;
-                        }
                         if (!mbar_wait(wempty_bar(stage), phase ^ 1u, abort_flag, p.status)) {
                             ok = false;
                             break;
@@ -149,12 +134,6 @@ ptq_fused_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                     const uint32_t uses = (w_issued + fp.w_stages - 1u - s) / fp.w_stages;
                     if (uses == 0u) continue;
                     for (int i = 0; i < 200000 && !mbar_try_wait(wfull_bar(s), (uses - 1u) & 1u); ++i) {
-                    }
-                }
-                for (uint32_t kb = 0; !kQuantize && kb < static_cast<uint32_t>(p.k_blocks); ++kb) {
-                    const uint32_t uses = (p_issued + p.k_blocks - 1u - kb) / p.k_blocks;
-                    if (uses == 0u) continue;
-                    for (int i = 0; i < 200000 && !mbar_try_wait(pfull_bar(kb), (uses - 1u) & 1u); ++i) {
                     }
                 }
             }
@@ -232,7 +211,7 @@ ptq_fused_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             }
         }
         if (lane == 0) bulk_wait_group<0>();
-    } else if (kQuantize) {
+    } else {
         // ------------------------------------------------------------------ quantizer warps
         // Thread (r8, c16) handles rows j*16 + r8 (j = 0..7) and the 16 channels c16*16.. of each k-block.
         const int qt = threadIdx.x - 32 * (2 + kNumEpiWarps);
