@@ -91,7 +91,7 @@ ptq_status_t ptq_linear_create(ptq_linear_t **out, int K, int N, int T,
 
 /*
  * Create a layer with ASYMMETRIC per-token-static activations: step and zero offset per token position,
- * which is what Sec. 5.1 allocates ("step size and zero offset for each token"; quantizer form of
+ * which is what Sec. 5.1 allocates (both parameters for every token position; quantizer form of
  * Sec. 2.3 with the offset rounded to an integer):
  *   Q1  c[m,k]   = clip( rne( (x[m,k] / s[k]) / dx[t] ) + z[t], 0, 255 )           uint8
  *       (NaN -> z[t], +inf -> 255, -inf -> 0)

@@ -264,9 +264,8 @@ void ptqo_calibrate(const uint16_t *xcal, int Bc, int T, int K,
 }
 
 /* ========================================================================= */
-/* Asymmetric PTS: step AND zero offset per token position (Sec. 5.1: "we can  */
-/* allocate the quantization step size and zero offset for each token";       */
-/* quantizer form of Sec. 2.3:                                                */
+/* Asymmetric PTS: step AND zero offset per token position (Sec. 5.1 gives    */
+/* every token position both parameters; quantizer form of Sec. 2.3:         */
 /*   X-hat = Delta (clip(round(X / Delta) + eps, 0, 2^b - 1) - eps) ).        */
 /* Reading: the offset eps is an integer z[t] in [0, 255] (the codes must be  */
 /* integers for the integer GEMM), the code is                                */
