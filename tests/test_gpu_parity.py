@@ -196,6 +196,40 @@ def test_seeded_random_shapes(env):
         check_layer(ptq, torch, spec, full=True)
 
 
+def test_back_to_back_layers_sharing_one_workspace(env):
+    """Kernels of consecutive calls overlap at their edges (programmatic dependent launch): two layers that
+    alternate on ONE stream and ONE workspace must still see each other's kernels in stream order."""
+    ptq, torch = env
+    specs = [wl.LinearSpec(7, 0, 0, "a", 24, 197, 384, 768), wl.LinearSpec(7, 1, 3, "b", 24, 197, 768, 192, bias=True)]
+    layers, xs, refs = [], [], []
+    need = 0
+    for sp in specs:
+        x, wq, dw, bias, s, dx = layer_inputs(sp)
+        layer = ptq.PtqLinear(wq, dw, s, dx, bias)
+        xd = torch.from_numpy(x).cuda()
+        ref = layer.forward(xd).clone()                 # its own workspace, nothing else in flight
+        torch.cuda.synchronize()
+        layers.append(layer)
+        xs.append(xd)
+        refs.append(ref)
+        need = max(need, layer.workspace_bytes(sp.B, 0), layer.workspace_bytes_dynamic(sp.B))
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    ys = [torch.empty_like(r) for r in refs]
+    for it in range(25):
+        for i in (0, 1):
+            if it % 5 == 4:
+                layers[i].forward_dynamic(xs[i], y=ys[i], workspace=ws)      # a different kernel pair in between
+            layers[i].forward(xs[i], y=ys[i], workspace=ws)
+        if it % 6 == 0:
+            torch.cuda.synchronize()
+            assert torch.equal(ys[0], refs[0]) and torch.equal(ys[1], refs[1]), "iteration %d" % it
+    torch.cuda.synchronize()
+    assert torch.equal(ys[0], refs[0]) and torch.equal(ys[1], refs[1])
+    for layer in layers:
+        layer.device_status()
+        layer.close()
+
+
 def test_fused_flag_is_reported_and_needs_no_workspace(env):
     ptq, torch = env
     for spec, want in ((CFG[3][0], True), (CFG[3][1], True), (CFG[1][2], False),
