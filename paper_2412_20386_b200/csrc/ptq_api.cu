@@ -148,20 +148,36 @@ ptq_status_t check_device(const ptq_linear *h)
     return PTQ_OK;
 }
 
-template <typename Kern>
-ptq_status_t ensure_smem(Kern kern, int bytes)
+// Opt a kernel in to `bytes` of dynamic shared memory, once per kernel and device (the attribute belongs
+// to the function on the CURRENT device, which the callers have checked to be `device`).  The kernel is
+// a template argument so that every kernel has its own flags.
+template <auto kKern>
+ptq_status_t ensure_smem(int device, int bytes)
 {
-    PTQ_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+    constexpr int kMaxDevices = 64;
+    static std::mutex mu;
+    static bool done[kMaxDevices] = {};
+    if (device < 0 || device >= kMaxDevices) return fail(PTQ_ERR_CUDA, "device index %d out of range", device);
+    std::lock_guard<std::mutex> lock(mu);
+    if (!done[device]) {
+        PTQ_CUDA(cudaFuncSetAttribute(kKern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+        done[device] = true;
+    }
     return PTQ_OK;
 }
 
 // How many 2-CTA clusters of the pair kernel can be resident at once (0 if cluster launch is unavailable).
-int query_max_pairs()
+int query_max_pairs(int device)
 {
-    static int cached = -1;
+    constexpr int kMaxDevices = 64;
+    static int cache[kMaxDevices];
+    static bool known[kMaxDevices] = {};
     static std::mutex mu;
+    if (device < 0 || device >= kMaxDevices) return 0;
     std::lock_guard<std::mutex> lock(mu);
-    if (cached >= 0) return cached;
+    if (known[device]) return cache[device];
+    known[device] = true;                      // per device: attributes and occupancy belong to the current device
+    int &cached = cache[device];
     cached = 0;
     if (cudaFuncSetAttribute(ptq::ptq_gemm_dequant_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              ptq::kPairSmemBytes) != cudaSuccess ||
@@ -323,12 +339,8 @@ ptq_status_t launch_quantize_dynamic(const ptq_linear *h, const void *x, long lo
 ptq_status_t launch_gemm(const ptq_linear *h, const void *codes, long long M, void *y, void *acc_out,
                          cudaStream_t stream, bool want_pair = false, const float *dx_rows = nullptr)
 {
-    static std::once_flag once;
-    static ptq_status_t attr_status = PTQ_OK;
-    std::call_once(once, [] {
-        attr_status = ensure_smem(ptq::ptq_gemm_dequant_kernel<false>, ptq::kGemmSmemBytes);
-        if (attr_status == PTQ_OK) attr_status = ensure_smem(ptq::ptq_gemm_dequant_kernel<true>, ptq::kGemmSmemBytes);
-    });
+    ptq_status_t attr_status = ensure_smem<ptq::ptq_gemm_dequant_kernel<false>>(h->device, ptq::kGemmSmemBytes);
+    if (attr_status == PTQ_OK) attr_status = ensure_smem<ptq::ptq_gemm_dequant_kernel<true>>(h->device, ptq::kGemmSmemBytes);
     if (attr_status != PTQ_OK) return attr_status;
 
     CUtensorMap tmA, tmY;
@@ -433,12 +445,13 @@ void choose_astat(ptq_linear *h)
     }
 }
 
-template <typename Kern>
-ptq_status_t launch_fused_kernel(Kern kern, const ptq_linear *h, const CUtensorMap &tmY, const ptq::FusedParams &fp,
-                                 int grid, cudaStream_t stream)
+template <auto kKern>
+ptq_status_t launch_fused_kernel(const ptq_linear *h, const CUtensorMap &tmY, const ptq::FusedParams &fp, int grid,
+                                 cudaStream_t stream)
 {
-    PTQ_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ptq::kFusedSmemLimit));
-    kern<<<grid, ptq::kFusedThreadsQuant, h->as_smem, stream>>>(h->tmWas, tmY, fp);
+    const ptq_status_t attr_status = ensure_smem<kKern>(h->device, ptq::kFusedSmemLimit);
+    if (attr_status != PTQ_OK) return attr_status;
+    kKern<<<grid, ptq::kFusedThreadsQuant, h->as_smem, stream>>>(h->tmWas, tmY, fp);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     PTQ_CUDA(cudaGetLastError());
     return PTQ_OK;
@@ -491,10 +504,10 @@ ptq_status_t launch_fused(const ptq_linear *h, const void *x, long long M, void 
     const int grid = p.m_tiles < h->num_sms ? p.m_tiles : h->num_sms;
     const bool dbg = acc_out != nullptr;
     if (h->fast_div)
-        return dbg ? launch_fused_kernel(ptq::ptq_fused_linear_kernel<true, true>, h, tmY, fp, grid, stream)
-                   : launch_fused_kernel(ptq::ptq_fused_linear_kernel<true, false>, h, tmY, fp, grid, stream);
-    return dbg ? launch_fused_kernel(ptq::ptq_fused_linear_kernel<false, true>, h, tmY, fp, grid, stream)
-               : launch_fused_kernel(ptq::ptq_fused_linear_kernel<false, false>, h, tmY, fp, grid, stream);
+        return dbg ? launch_fused_kernel<ptq::ptq_fused_linear_kernel<true, true>>(h, tmY, fp, grid, stream)
+                   : launch_fused_kernel<ptq::ptq_fused_linear_kernel<true, false>>(h, tmY, fp, grid, stream);
+    return dbg ? launch_fused_kernel<ptq::ptq_fused_linear_kernel<false, true>>(h, tmY, fp, grid, stream)
+               : launch_fused_kernel<ptq::ptq_fused_linear_kernel<false, false>>(h, tmY, fp, grid, stream);
 }
 
 bool fused_usable(const ptq_linear *h) { return h->as_ok && h->K % 16 == 0; }
@@ -688,7 +701,7 @@ static ptq_status_t create_impl(ptq_linear_t **out, int K, int N, int T, const i
                          static_cast<unsigned long long>(Npad), static_cast<unsigned long long>(h->Kpad), ptq::kBK,
                          static_cast<unsigned>(h->BN / 2));
         if (st != PTQ_OK) break;
-        h->max_pairs = h->asym ? 0 : query_max_pairs();
+        h->max_pairs = h->asym ? 0 : query_max_pairs(dev);
         if (h->as_ok)
             st = make_map_2d(&h->tmWas, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, h->d_w, static_cast<unsigned long long>(K),
                              static_cast<unsigned long long>(Npad), static_cast<unsigned long long>(h->Kpad),
