@@ -36,6 +36,8 @@ if ROOT not in sys.path:
 METRIC = "PTS W8A8 linear INT8 TOPS (quant+GEMM+dequant)"
 UNIT = "TOPS"
 INT8_OVER_BF16 = 2.0          # nominal dense ratio 4.5 / 2.25 PFLOP/s
+INT8_NOMINAL_TOPS = 4500.0    # dense INT8 peak of one B200 (vendor datasheet)
+SUSTAIN_SECONDS = 1.0         # length of the sustained leg; also the region length from which the sustained peak applies
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -89,38 +91,45 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.lines.append((time.time(), line.strip()))
 
-    def stop(self, t0=None, t1=None, t2=None):
-        """Summarise the samples taken in [t0, t1] (the timed region); if fewer than three fall inside
-        it, widen to [t0, t2] (the end-to-end loop that follows, same kernels) and say so."""
+    def stop(self, t0, t1, s0, s1):
+        """Two summaries: the samples taken in [t0, t1] (the headline region) and in [s0, s1] (the
+        sustained leg).  A headline region too short to hold three samples takes the sustained leg's
+        clocks (same kernels, longer run) and says so in `window`."""
+        empty = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+            return dict(empty), dict(empty)
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
-        window = "timed region"
-        lines = [l for (ts, l) in self.lines if t0 is None or (t0 <= ts <= t1)]
-        if t0 is not None and len(lines) < 3:
-            lines = [l for (ts, l) in self.lines if t0 <= ts <= (t2 or t1)]
-            window = "timed region + end-to-end loop"
-        sm, smax, reasons = [], [], set()
-        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
-        for line in lines:
-            parts = [p.strip() for p in line.split(",")]
-            if len(parts) < 6:
-                continue
-            try:
-                sm.append(float(parts[0]))
-                smax.append(float(parts[1]))
-            except ValueError:
-                continue
-            for n, v in zip(names, parts[2:6]):
-                if v.lower().startswith("active"):
-                    reasons.add(n)
-        return {"sm_mhz": statistics.median(sm) if sm else None,
-                "sm_max_mhz": max(smax) if smax else None,
-                "reasons": sorted(reasons), "samples": len(sm), "window": window}
+
+        def summary(a, b):
+            sm, smax, reasons = [], [], set()
+            names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+            for ts, line in self.lines:
+                if not (a <= ts <= b):
+                    continue
+                parts = [p.strip() for p in line.split(",")]
+                if len(parts) < 6:
+                    continue
+                try:
+                    sm.append(float(parts[0]))
+                    smax.append(float(parts[1]))
+                except ValueError:
+                    continue
+                for n, v in zip(names, parts[2:6]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+            return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                    "reasons": sorted(reasons), "samples": len(sm)}
+
+        head, sus = summary(t0, t1), summary(s0, s1)
+        head["window"] = "timed region"
+        if head["samples"] < 3:
+            head = dict(sus)
+            head["window"] = "sustained leg (the timed region is shorter than three 50 ms samples)"
+        return head, sus
 
 
 # ------------------------------------------------------------------------------------------------
@@ -240,6 +249,17 @@ def reduce_max_over_ranks(values, device=None):
     return [float(v) for v in t]
 
 
+def pct_of_peak(tops_per_gpu, region_seconds, int8_burst, int8_sustained):
+    """Per-GPU throughput as a percentage of the nominal dense INT8 peak and of the measured proxy that
+    fits the length of the timed region: 2 x bf16 burst below SUSTAIN_SECONDS, 2 x bf16 sustained from there."""
+    long_run = region_seconds >= SUSTAIN_SECONDS
+    proxy = int8_sustained if long_run else int8_burst
+    return {"nominal_4500": 100.0 * tops_per_gpu / INT8_NOMINAL_TOPS,
+            "measured_proxy": 100.0 * tops_per_gpu / proxy,
+            "proxy": "2 x bf16_tflops%s = %.0f TOPS (timed region %.3f s)" % ("_sustained" if long_run else "", proxy,
+                                                                             region_seconds)}
+
+
 def whole_job_tops(world, step_ops_per_rank, ms_per_step):
     """Replicas: every rank does step_ops_per_rank in the (max over ranks) step time."""
     return world * step_ops_per_rank / (ms_per_step * 1e-3) / 1e12
@@ -292,7 +312,8 @@ def run_ours(args, specs, rank, world, local_rank):
             s, dx, z = ptq.calibrate_asym(xcal, wq, dw)          # Q0 on the GPU, with zero offsets
             layer = ptq.PtqLinear(wq, dw, s, dx, bias, act_zero=z)
         else:
-            s, dx = ptq.calibrate(xcal, wq, dw)                  # Q0 on the GPU
+            # Q0 on the GPU; `static` is the per-tensor comparator: one step for all token positions
+            s, dx = ptq.calibrate(xcal, wq, dw, per_tensor=(args.scheme == "static"))
             layer = ptq.PtqLinear(wq, dw, s, dx, bias)
         x_dev = x_host.to(dev)
         y_dev = torch.empty((sp.B, sp.T, sp.N), dtype=torch.float16, device=dev)
@@ -373,6 +394,10 @@ def run_ours(args, specs, rank, world, local_rank):
         step = graph.replay
 
     # ---- device-resident timing -------------------------------------------------------------
+    # (1) the headline: exactly `steps` steps between one event pair; (2) the same steps again, each with
+    # its own event pair (median and minimum, the protocol of the paper's Appendix B.2); (3) a sustained
+    # leg: the step repeated for at least SUSTAIN_SECONDS, long enough for the clock samples (every
+    # 50 ms) to fall inside it and for the power cap to act, reported beside the headline.
     for _ in range(args.warmup):
         step()
     barrier()
@@ -395,6 +420,21 @@ def run_ours(args, specs, rank, world, local_rank):
     for d in layers:
         d["layer"].device_status()
 
+    n_each = max(3, min(args.steps, 200))
+    _, step_min, step_med = event_times_ms(torch, step, n_each)
+
+    n_sus = int(min(200000, max(args.steps, SUSTAIN_SECONDS * 1e3 / max(ms_total / args.steps, 1e-4))))
+    g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ts0 = time.time()
+    g0.record()
+    for _ in range(n_sus):
+        step()
+    g1.record()
+    barrier()
+    ts1 = time.time()
+    ms_sus = g0.elapsed_time(g1) / n_sus
+
     # ---- end to end with host buffers -------------------------------------------------------
     for _ in range(min(args.warmup, 3)):
         step_e2e()
@@ -409,9 +449,9 @@ def run_ours(args, specs, rank, world, local_rank):
     f1.record()
     barrier()
     ms_e2e = f0.elapsed_time(f1) / e2e_steps
-    clocks = sampler.stop(t_start, t_end, time.time())
+    clocks, clocks_sus = sampler.stop(t_start, t_end, ts0, ts1)
 
-    ms_total, ms_e2e = reduce_max_over_ranks([ms_total, ms_e2e], dev)
+    ms_total, ms_e2e, ms_sus = reduce_max_over_ranks([ms_total, ms_e2e, ms_sus], dev)
     ms_step = ms_total / args.steps
     value = whole_job_tops(world, step_ops, ms_step)
     e2e_value = whole_job_tops(world, step_ops, ms_e2e)
@@ -420,7 +460,11 @@ def run_ours(args, specs, rank, world, local_rank):
         return
 
     # ---- per-kernel timing (rank 0): each kernel alone, events around every launch ----------
-    int8_peak = peaks["bf16_tflops_sustained"] * INT8_OVER_BF16
+    # Kernels timed alone (50 launches, a few milliseconds, full clock) are rated against the BURST proxy
+    # 2 x bf16_tflops; the sustained proxy applies only to regions of a second or more.
+    int8_burst = peaks["bf16_tflops"] * INT8_OVER_BF16
+    int8_sustained = peaks["bf16_tflops_sustained"] * INT8_OVER_BF16
+    int8_peak = int8_burst
     hbm_peak = peaks["hbm_gbs"]
     kernels = []
     iters = 50
@@ -478,6 +522,7 @@ def run_ours(args, specs, rank, world, local_rank):
         k["tops"] = k["ops"] / t / 1e12
         k["gbs"] = k["bytes"] / t / 1e9
         k["frac_tensor"] = k["tops"] / int8_peak
+        k["frac_tensor_nominal"] = k["tops"] / INT8_NOMINAL_TOPS
         k["frac_hbm"] = k["gbs"] / hbm_peak
         k["bound"] = "tensor" if k["frac_tensor"] >= k["frac_hbm"] else "hbm"
     # the dominant kernel is the one with the largest share of the step when timed alone
@@ -489,12 +534,12 @@ def run_ours(args, specs, rank, world, local_rank):
     dom = max((k for k in kernels if k["kernel"] == dom_name), key=lambda k: k["ms"])
     if dom["bound"] == "tensor":
         roof = {"bound": "tensor", "achieved": dom["tops"], "peak": int8_peak, "unit": "TFLOP/s",
-                "frac": dom["frac_tensor"]}
+                "frac": dom["frac_tensor"], "frac_of_nominal_4500": dom["frac_tensor_nominal"]}
     else:
         roof = {"bound": "hbm", "achieved": dom["gbs"], "peak": hbm_peak, "unit": "GB/s", "frac": dom["frac_hbm"]}
     roof.update({"kernel": dom["kernel"], "layer": dom["layer"], "ms_per_launch": dom["ms"],
-                 "peak_source": "%s (%s)" % (("2 x bf16_tflops_sustained" if dom["bound"] == "tensor" else "hbm_gbs"),
-                                             peaks_kind),
+                 "peak_source": "%s (%s)" % (("2 x bf16_tflops, the burst figure: the kernel is timed alone over %d launches"
+                                              % iters if dom["bound"] == "tensor" else "hbm_gbs"), peaks_kind),
                  "traffic": TRAFFIC.get((dom["kernel"], args.workload, dom["layer"].split(".")[-1]))
                  if args.scheme == "pts" else None})
 
@@ -518,9 +563,16 @@ def run_ours(args, specs, rank, world, local_rank):
                    "l2": "inputs_larger_than_l2 (%.0f MB touched per step)" % (touched / 1e6)
                    if touched > 2 * 126e6 else "working set %.0f MB fits L2: L2-warm timing" % (touched / 1e6),
                    "parallelism": "replicas x%d" % world},
-        "pct_of_int8_peak": {"nominal_4500": 100.0 * value / world / 4500.0,
-                             "measured_2x_bf16_sustained": 100.0 * value / world / int8_peak},
+        "ms_per_step_median": step_med, "ms_per_step_min": step_min,
+        "pct_of_int8_peak": pct_of_peak(value / world, ms_total * 1e-3, int8_burst, int8_sustained),
         "clocks": clocks,
+        "sustained": {"seconds": round(ms_sus * n_sus * 1e-3, 3), "steps": n_sus, "ms_per_step": ms_sus,
+                      "value": whole_job_tops(world, step_ops, ms_sus), "unit": UNIT,
+                      "pct_of_int8_peak": pct_of_peak(whole_job_tops(1, step_ops, ms_sus), ms_sus * n_sus * 1e-3,
+                                                      int8_burst, int8_sustained),
+                      "clocks": clocks_sus,
+                      "ms_x_mhz": (ms_sus * clocks_sus["sm_mhz"]) if clocks_sus.get("sm_mhz") else None,
+                      "headline_ms_x_max_mhz": (ms_step * clocks_sus["sm_max_mhz"]) if clocks_sus.get("sm_max_mhz") else None},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": ms_e2e},
         "gpu_launches": int(launches),
@@ -544,15 +596,16 @@ TRAFFIC = {
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c3", choices=["c0", "c1", "c2", "c3", "c4"])
     ap.add_argument("--path", default="unfused", choices=["unfused", "fused", "pair"],
                     help="unfused: quantize kernel + GEMM kernel (fastest at present, the default); "
                          "fused: PTQ_FLAG_FUSED_PROLOGUE; pair: PTQ_FLAG_CTA_PAIR")
-    ap.add_argument("--scheme", default="pts", choices=["pts", "pts-asym", "dynamic", "w4a4"],
-                    help="pts: symmetric per-token-static codes (the default); pts-asym: with a zero offset per token "
+    ap.add_argument("--scheme", default="pts", choices=["pts", "static", "pts-asym", "dynamic", "w4a4"],
+                    help="pts: symmetric per-token-static codes (the default); static: the per-tensor static comparator "
+                         "(one step for the whole tensor, same kernels); pts-asym: with a zero offset per token "
                          "position; dynamic: the per-token dynamic comparator (row steps measured at run time); "
                          "w4a4: 4-bit codes and packed 4-bit weights on the 8-bit tensor-core path")
     ap.add_argument("--graph", action="store_true",

@@ -236,6 +236,18 @@ ptq_status_t ptq_calibrate(int K, int N, int T, const void *xcal_fp16, int Bc,
                            float *smooth_out, float *act_step_out, void *stream);
 
 /*
+ * Comparator: per-TENSOR static quantization (the coarsest granularity of the latency table of Sec. 6
+ * and of Fig. 5: one step for the whole activation tensor).  Same s[k] as ptq_calibrate, and
+ *   step = max( max_{b,t,k} |xcal[b,t,k] / s[k]|, 1e-5 ) / 127
+ * written to all T entries of act_step_out, so that the result feeds ptq_linear_create unchanged: a
+ * per-tensor static layer is a PTS layer whose steps are all equal and runs the same kernels.
+ * Arguments, ownership and errors as for ptq_calibrate.
+ */
+ptq_status_t ptq_calibrate_per_tensor(int K, int N, int T, const void *xcal_fp16, int Bc,
+                                      const int8_t *w_q, const float *w_step,
+                                      float *smooth_out, float *act_step_out, void *stream);
+
+/*
  * W4A4 layers (the bit width of the paper's latency table; Appendix B.1, quantization part).  The
  * arithmetic is that of ptq_linear_create / ptq_linear_forward with the signed 4-bit range:
  *     q = clamp(rne((x / s[k]) / act_step[t]), -8, 7),   acc = sum_k q * w4,   y as before,
@@ -307,6 +319,22 @@ ptq_status_t ptq_calibrate_asym(int K, int N, int T, const void *xcal_fp16, int 
  * call (its output is then undefined), or PTQ_ERR_CUDA.
  */
 ptq_status_t ptq_linear_device_status(const ptq_linear_t *h);
+
+/*
+ * Self-test of the failure path (no counterpart in the paper).  Every wait inside the kernels is
+ * bounded: a wait that does not end sets the handle's status word and the CTA unwinds.  This call
+ * makes that happen safely: it launches one tiny kernel that waits, for at most limit_us microseconds,
+ * on a barrier that nothing ever signals and that no copy or tensor-core operation refers to, gives
+ * up, and returns normally.  Afterwards ptq_linear_device_status(h) reports PTQ_ERR_TIMEOUT once and
+ * PTQ_OK from then on, and the handle keeps working.
+ *   limit_us   1 .. 100000
+ *   result3    host, 3 words: what the short wait and a second, long wait on the same barrier
+ *              returned (0 = gave up; the second leaves through the CTA-wide abort flag), and the
+ *              nanoseconds the second one waited
+ * Allocates 12 bytes of temporary device memory and synchronises the stream.
+ */
+ptq_status_t ptq_linear_selftest_wait_timeout(const ptq_linear_t *h, unsigned limit_us, unsigned *result3,
+                                              void *stream);
 
 /*
  * Write a one-line, human-readable description of the kernels and tilings chosen for this layer

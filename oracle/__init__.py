@@ -61,6 +61,8 @@ def _bind(path: str) -> ctypes.CDLL:
                                            vp, vp, vp, vp, vp, vp, vp, vp]
     L.ptqo_calibrate.restype = None
     L.ptqo_calibrate.argtypes = [vp, c_int, c_int, c_int, vp, vp, c_int, vp, vp]
+    L.ptqo_calibrate_per_tensor.restype = None
+    L.ptqo_calibrate_per_tensor.argtypes = [vp, c_int, c_int, c_int, vp, vp, c_int, vp, vp]
     L.ptqo_quantize4_one.restype = ctypes.c_int8
     L.ptqo_quantize4_one.argtypes = [ctypes.c_uint16, ctypes.c_float, ctypes.c_float]
     L.ptqo_quantize4.restype = None
@@ -231,6 +233,20 @@ def calibrate(xcal, wq, dw):
     dx = np.empty(T, np.float32)
     lib().ptqo_calibrate(_p(xcal), Bc, T, K, _p(wq), _p(dw), N, _p(s), _p(dx))
     return s, dx
+
+
+def calibrate_per_tensor(xcal, wq, dw):
+    """Per-tensor static comparator: (s fp32 [K], delta) with ONE activation step for all token positions."""
+    xcal = _c(xcal, np.float16)
+    Bc, T, K = xcal.shape
+    wq = _c(wq, np.int8)
+    N = wq.shape[0]
+    assert wq.shape == (N, K)
+    dw = _c(dw, np.float32)
+    s = np.empty(K, np.float32)
+    delta = np.empty(1, np.float32)
+    lib().ptqo_calibrate_per_tensor(_p(xcal), Bc, T, K, _p(wq), _p(dw), N, _p(s), _p(delta))
+    return s, np.float32(delta[0])
 
 
 # --------------------------------------------------------------------------- #

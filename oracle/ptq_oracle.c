@@ -263,6 +263,37 @@ void ptqo_calibrate(const uint16_t *xcal, int Bc, int T, int K,
     }
 }
 
+/* Per-tensor static comparator (the coarsest granularity in the latency      */
+/* table of Sec. 6 and in Fig. 5): the smoothing scales of ptqo_calibrate and */
+/* ONE step for the whole activation tensor,                                  */
+/*   delta = max( max_{b,t,k} |x[b,t,k] / s[k]|, 1e-5 ) / 127,                */
+/* i.e. the min-max rule of Sec. 2.3 taken over every token position at once. */
+/* Pinned: numpy float32; equals the largest per-position step; never clips   */
+/* the calibration batch; degenerate (all-zero) batch gives the floor.        */
+void ptqo_calibrate_per_tensor(const uint16_t *xcal, int Bc, int T, int K,
+                               const int8_t *wq, const float *dw, int N,
+                               float *s, float *delta)
+{
+    const float floor_ = 1e-5f;
+    long M = (long)Bc * T, m;
+    int k;
+    float mu = 0.0f;
+    float *dx_pos = (float *)malloc(sizeof(float) * (size_t)T);
+    ptqo_calibrate(xcal, Bc, T, K, wq, dw, N, s, dx_pos);    /* s only; the per-position steps are discarded */
+    free(dx_pos);
+    for (m = 0; m < M; ++m)
+        for (k = 0; k < K; ++k) {
+            volatile float u = ptqo_half_to_float(xcal[m * K + k]) / s[k];
+            float a = fabsf(u);
+            if (a > mu) mu = a;
+        }
+    if (mu < floor_) mu = floor_;
+    {
+        volatile float d = mu / 127.0f;
+        *delta = d;
+    }
+}
+
 /* ========================================================================= */
 /* Asymmetric PTS: step AND zero offset per token position (Sec. 5.1 gives    */
 /* every token position both parameters; quantizer form of Sec. 2.3:         */

@@ -84,6 +84,10 @@ def load_library() -> ctypes.CDLL:
     L.ptq_calibrate.argtypes = [ci, ci, ci, vp, ci, vp, vp, vp, vp, vp]
     L.ptq_linear_create_w4a4.restype = ci
     L.ptq_linear_create_w4a4.argtypes = [ctypes.POINTER(vp), ci, ci, ci, vp, vp, vp, vp, vp, cu]
+    L.ptq_linear_selftest_wait_timeout.restype = ci
+    L.ptq_linear_selftest_wait_timeout.argtypes = [vp, ctypes.c_uint, vp, vp]
+    L.ptq_calibrate_per_tensor.restype = ci
+    L.ptq_calibrate_per_tensor.argtypes = [ci, ci, ci, vp, ci, vp, vp, vp, vp, vp]
     L.ptq_calibrate_w4a4.restype = ci
     L.ptq_calibrate_w4a4.argtypes = [ci, ci, ci, vp, ci, vp, vp, vp, vp, vp]
     L.ptq_quantize_packed4.restype = ci
@@ -127,6 +131,17 @@ def _stream_ptr(stream) -> Optional[int]:
         import torch
         stream = torch.cuda.current_stream()
     return ctypes.c_void_p(int(stream.cuda_stream))
+
+
+def _scratch(nbytes: int, device, stream):
+    """A temporary device buffer for one call.  The kernels run on `stream`, which need not be the
+    stream torch's allocator associates the block with: recording the use keeps the block from being
+    handed out again while the kernels still read it."""
+    import torch
+    buf = torch.empty(max(int(nbytes), 16), dtype=torch.uint8, device=device)
+    if stream is not None:
+        buf.record_stream(stream)
+    return buf
 
 
 def kernel_launch_count() -> int:
@@ -197,6 +212,12 @@ class PtqLinear:
     def device_status(self):
         _check(self._L.ptq_linear_device_status(self._h))
 
+    def selftest_wait_timeout(self, limit_us: int = 50, stream=None):
+        """``ptq_linear_selftest_wait_timeout``: returns (short wait result, long wait result, ns waited)."""
+        out = (ctypes.c_uint * 3)()
+        _check(self._L.ptq_linear_selftest_wait_timeout(self._h, int(limit_us), out, _stream_ptr(stream)))
+        return int(out[0]), int(out[1]), int(out[2])
+
     # -- calls -----------------------------------------------------------------
     def _batch(self, x):
         import torch
@@ -212,9 +233,12 @@ class PtqLinear:
         B = self._batch(x)
         if y is None:
             y = torch.empty((B, self.T, self.N), dtype=torch.float16, device=x.device)
-        need = self.workspace_bytes(B, flags)
+        if flags & FLAG_FUSED_PROLOGUE and x.data_ptr() % 16:
+            need = self.workspace_bytes(B, 0)      # an x that is not 16-byte aligned takes the two-kernel path
+        else:
+            need = self.workspace_bytes(B, flags)
         if workspace is None and need:
-            workspace = torch.empty(need, dtype=torch.uint8, device=x.device)
+            workspace = _scratch(need, x.device, stream)
         wptr = workspace.data_ptr() if workspace is not None else None
         wbytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
         _check(self._L.ptq_linear_forward(self._h, x.data_ptr(), B, y.data_ptr(), wptr, wbytes,
@@ -243,7 +267,7 @@ class PtqLinear:
         if y is None:
             y = torch.empty((B, self.T, self.N), dtype=torch.float16, device=x.device)
         if workspace is None:
-            workspace = torch.empty(self.workspace_bytes_dynamic(B), dtype=torch.uint8, device=x.device)
+            workspace = _scratch(self.workspace_bytes_dynamic(B), x.device, stream)
         _check(self._L.ptq_linear_forward_dynamic(self._h, x.data_ptr(), B, y.data_ptr(), workspace.data_ptr(),
                                                   workspace.numel() * workspace.element_size(),
                                                   _stream_ptr(stream)))
@@ -259,7 +283,7 @@ class PtqLinear:
         acc = torch.empty((B, self.T, self.N), dtype=torch.int32, device=dev)
         step = torch.empty(B * self.T, dtype=torch.float32, device=dev)
         need = self.workspace_bytes_dynamic(B)
-        ws = torch.empty(need, dtype=torch.uint8, device=dev)
+        ws = _scratch(need, dev, stream)
         _check(self._L.ptq_linear_forward_dynamic_debug(self._h, x.data_ptr(), B, y.data_ptr(), q.data_ptr(),
                                                         acc.data_ptr(), step.data_ptr(), ws.data_ptr(), need,
                                                         _stream_ptr(stream)))
@@ -280,7 +304,7 @@ class PtqLinear:
         B = self._batch(x)
         out = torch.empty((B, self.T, (self.K + 1) // 2), dtype=torch.uint8, device=x.device)
         need = self.workspace_bytes(B, 0)
-        ws = torch.empty(need, dtype=torch.uint8, device=x.device)
+        ws = _scratch(need, x.device, stream)
         _check(self._L.ptq_quantize_packed4(self._h, x.data_ptr(), B, out.data_ptr(), ws.data_ptr(), need,
                                             _stream_ptr(stream)))
         return out
@@ -310,7 +334,7 @@ class PtqLinear:
                         device=dev) if want_q else None
         acc = torch.empty((B, self.T, self.N), dtype=torch.int32, device=dev) if want_acc else None
         need = self.workspace_bytes(B, 0)
-        ws = torch.empty(need, dtype=torch.uint8, device=dev)
+        ws = _scratch(need, dev, stream)
         _check(self._L.ptq_linear_forward_debug(
             self._h, x.data_ptr(), B, y.data_ptr(),
             q.data_ptr() if q is not None else None,
@@ -319,8 +343,9 @@ class PtqLinear:
         return y, q, acc
 
 
-def calibrate(xcal, w_q, w_step, stream=None):
-    """``ptq_calibrate``: device fp16 [Bc,T,K] -> (s fp32 [K], dx fp32 [T]) as numpy arrays."""
+def calibrate(xcal, w_q, w_step, stream=None, per_tensor: bool = False):
+    """``ptq_calibrate``: device fp16 [Bc,T,K] -> (s fp32 [K], dx fp32 [T]) as numpy arrays.
+    ``per_tensor=True`` calls ``ptq_calibrate_per_tensor`` (one step, repeated T times)."""
     import torch
     L = load_library()
     if xcal.dtype != torch.float16 or not xcal.is_cuda or not xcal.is_contiguous() or xcal.dim() != 3:
@@ -333,8 +358,8 @@ def calibrate(xcal, w_q, w_step, stream=None):
     w_step = _host(w_step, np.float32, (N,))
     s = np.empty(K, np.float32)
     dx = np.empty(T, np.float32)
-    _check(L.ptq_calibrate(K, N, T, xcal.data_ptr(), Bc, _hp(w_q), _hp(w_step), _hp(s), _hp(dx),
-                           _stream_ptr(stream)))
+    fn = L.ptq_calibrate_per_tensor if per_tensor else L.ptq_calibrate
+    _check(fn(K, N, T, xcal.data_ptr(), Bc, _hp(w_q), _hp(w_step), _hp(s), _hp(dx), _stream_ptr(stream)))
     return s, dx
 
 

@@ -974,9 +974,33 @@ ptq_status_t ptq_linear_device_status(const ptq_linear_t *h)
     return PTQ_OK;
 }
 
+ptq_status_t ptq_linear_selftest_wait_timeout(const ptq_linear_t *h, unsigned limit_us, unsigned *result3, void *stream)
+{
+    if (!h || !result3) return fail(PTQ_ERR_NULL, "handle and result must not be NULL");
+    if (limit_us < 1 || limit_us > 100000) return fail(PTQ_ERR_VALUE, "limit_us must be in [1, 100000] (got %u)", limit_us);
+    ptq_status_t st = check_device(h);
+    if (st != PTQ_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    unsigned *d_out = nullptr;
+    PTQ_CUDA(cudaMalloc(reinterpret_cast<void **>(&d_out), 3 * sizeof(unsigned)));
+    auto body = [&]() -> ptq_status_t {
+        PTQ_CUDA(cudaMemsetAsync(d_out, 0xff, 3 * sizeof(unsigned), s));
+        ptq::ptq_wait_selftest_kernel<<<1, 64, 0, s>>>(h->d_status, 1000ull * limit_us, d_out);
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+        PTQ_CUDA(cudaGetLastError());
+        PTQ_CUDA(cudaMemcpyAsync(result3, d_out, 3 * sizeof(unsigned), cudaMemcpyDeviceToHost, s));
+        PTQ_CUDA(cudaStreamSynchronize(s));
+        return PTQ_OK;
+    };
+    st = body();
+    cudaFree(d_out);
+    return st;
+}
+
 static ptq_status_t calibrate_impl(int K, int N, int T, const void *xcal_fp16, int Bc, const int8_t *w_q,
                                    const float *w_step, float *smooth_out, float *act_step_out,
-                                   int32_t *act_zero_out, void *stream, float qmax = 127.0f)
+                                   int32_t *act_zero_out, void *stream, float qmax = 127.0f,
+                                   bool per_tensor = false)
 {
     if (!xcal_fp16 || !w_q || !w_step || !smooth_out || !act_step_out)
         return fail(PTQ_ERR_NULL, "calibrate: pointers must not be NULL");
@@ -1018,7 +1042,10 @@ static ptq_status_t calibrate_impl(int K, int N, int T, const void *xcal_fp16, i
                                                                            reinterpret_cast<int *>(d_out + K + T));
         } else {
             ptq::ptq_calib_rowmax_kernel<<<grid, 256, 0, s>>>(x, M, K, T, d_out, d_bits + K);
-            ptq::ptq_calib_step_kernel<<<(T + 127) / 128, 128, 0, s>>>(d_bits + K, T, d_out + K, qmax);
+            if (per_tensor)
+                ptq::ptq_calib_step_tensor_kernel<<<1, 256, 0, s>>>(d_bits + K, T, d_out + K, qmax);
+            else
+                ptq::ptq_calib_step_kernel<<<(T + 127) / 128, 128, 0, s>>>(d_bits + K, T, d_out + K, qmax);
         }
         g_launches.fetch_add(5, std::memory_order_relaxed);
         PTQ_CUDA(cudaGetLastError());
@@ -1041,6 +1068,12 @@ ptq_status_t ptq_calibrate(int K, int N, int T, const void *xcal_fp16, int Bc, c
                            const float *w_step, float *smooth_out, float *act_step_out, void *stream)
 {
     return calibrate_impl(K, N, T, xcal_fp16, Bc, w_q, w_step, smooth_out, act_step_out, nullptr, stream);
+}
+
+ptq_status_t ptq_calibrate_per_tensor(int K, int N, int T, const void *xcal_fp16, int Bc, const int8_t *w_q,
+                                      const float *w_step, float *smooth_out, float *act_step_out, void *stream)
+{
+    return calibrate_impl(K, N, T, xcal_fp16, Bc, w_q, w_step, smooth_out, act_step_out, nullptr, stream, 127.0f, true);
 }
 
 ptq_status_t ptq_calibrate_asym(int K, int N, int T, const void *xcal_fp16, int Bc, const int8_t *w_q,

@@ -109,6 +109,24 @@ __global__ void __launch_bounds__(128) ptq_calib_step_kernel(const unsigned *mu_
     dx[t] = __fdiv_rn(fmaxf(__uint_as_float(mu_bits[t]), kCalibFloor), qmax);      // 127 levels, or 7 for 4-bit codes
 }
 
+// Per-tensor static comparator: ONE step for every token position, from the largest smoothed magnitude
+// of the whole calibration batch, dx[t] = max(max_t mu[t], 1e-5) / 127 for all t.  One block.
+__global__ void __launch_bounds__(256) ptq_calib_step_tensor_kernel(const unsigned *mu_bits, int T, float *dx,
+                                                                    float qmax)
+{
+    __shared__ unsigned warp_best[8];
+    unsigned best = 0u;                                   // bit patterns of non-negative floats order like the floats
+    for (int t = threadIdx.x; t < T; t += blockDim.x) best = max(best, mu_bits[t]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) best = max(best, __shfl_xor_sync(0xffffffffu, best, o));
+    if ((threadIdx.x & 31) == 0) warp_best[threadIdx.x >> 5] = best;
+    __syncthreads();
+    best = warp_best[0];
+    for (int w = 1; w < static_cast<int>(blockDim.x >> 5); ++w) best = max(best, warp_best[w]);
+    const float step = __fdiv_rn(fmaxf(__uint_as_float(best), kCalibFloor), qmax);
+    for (int t = threadIdx.x; t < T; t += blockDim.x) dx[t] = step;
+}
+
 // --- asymmetric variant: per-token-position range [lo, hi] of x/s, always containing zero ----------
 //   hi[t] = max(0, max x/s),  nlo[t] = max(0, max -(x/s))   (both non-negative: atomicMax on the bits)
 //   dx[t] = max(hi + nlo, 1e-5) / 255,   z[t] = clip(rne(nlo / dx[t]), 0, 255)

@@ -77,7 +77,7 @@ constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 // Wait for the phase with the given parity.  `abort_flag` is a CTA-wide shared word: once any
 // thread has given up, every other wait in the CTA returns false at its next check.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag,
-                                          unsigned *status)
+                                          unsigned *status, unsigned long long limit_ns = kWaitLimitNs)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = global_timer_ns();
@@ -86,13 +86,42 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         if (mbar_try_wait(bar, parity)) return true;
         if ((++spins & 63u) == 0u) {
             if (*abort_flag) return false;
-            if (global_timer_ns() - t0 > kWaitLimitNs) {
+            if (global_timer_ns() - t0 > limit_ns) {
                 *abort_flag = 1u;
                 atomicOr(status, PTQ_DEV_TIMEOUT);
                 return false;
             }
         }
     }
+}
+
+// Self-test of the bounded wait, for the failure-detection tests: one CTA of 64 threads and one mbarrier
+// that nothing ever arrives on (no copy, no MMA and no other thread refers to it, so giving up leaves
+// nothing in flight).  Thread 0 waits with the short limit `limit_ns` and must give up: it raises the
+// CTA's abort flag and sets PTQ_DEV_TIMEOUT in `status`.  Thread 32 waits on the same barrier with the
+// ordinary long limit and must leave through the abort flag.  out[0], out[1]: what the two waits returned
+// (0 = gave up); out[2]: nanoseconds thread 32 spent waiting.
+__global__ void __launch_bounds__(64) ptq_wait_selftest_kernel(unsigned *status, unsigned long long limit_ns,
+                                                               unsigned *out)
+{
+    __shared__ __align__(8) unsigned long long bar;
+    __shared__ uint32_t abort_word;
+    const uint32_t bar_addr = smem_u32(&bar);
+    if (threadIdx.x == 0) {
+        mbar_init(bar_addr, 1);
+        abort_word = 0u;
+        fence_mbar_init();
+    }
+    __syncthreads();
+    volatile uint32_t *abort_flag = &abort_word;
+    if (threadIdx.x == 0) {
+        out[0] = mbar_wait(bar_addr, 0u, abort_flag, status, limit_ns) ? 1u : 0u;
+    } else if (threadIdx.x == 32) {
+        const unsigned long long t0 = global_timer_ns();
+        out[1] = mbar_wait(bar_addr, 0u, abort_flag, status) ? 1u : 0u;
+        out[2] = static_cast<unsigned>(global_timer_ns() - t0);
+    }
+    __syncthreads();
 }
 
 // ---------------------------------------------------------------- proxies / fences

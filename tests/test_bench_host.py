@@ -87,3 +87,38 @@ def test_oracle_sampling_plan_is_bounded():
     assert len(data) == 1 and 8 <= data[0][1] <= specs[0].M and "rows" in sample
     ops, secs = bench.run_oracle_pass(data)
     assert ops == 2.0 * data[0][1] * specs[0].K * specs[0].N and secs > 0
+
+
+def test_measured_proxy_follows_the_length_of_the_timed_region():
+    sys.path.insert(0, ROOT)
+    import bench
+    short = bench.pct_of_peak(1500.0, 0.005, 3312.0, 2744.0)
+    long_ = bench.pct_of_peak(1300.0, 1.2, 3312.0, 2744.0)
+    assert short["nominal_4500"] == pytest.approx(100 * 1500 / 4500)
+    assert short["measured_proxy"] == pytest.approx(100 * 1500 / 3312) and "sustained" not in short["proxy"]
+    assert long_["measured_proxy"] == pytest.approx(100 * 1300 / 2744) and "bf16_tflops_sustained" in long_["proxy"]
+
+
+def test_clock_summaries_keep_the_two_windows_apart():
+    sys.path.insert(0, ROOT)
+    import bench
+
+    class FakeProc:
+        def terminate(self):
+            pass
+
+        def wait(self, timeout=None):
+            return 0
+
+    smp = bench.ClockSampler(0)
+    smp.proc = FakeProc()
+    line = lambda mhz, cap: "%d, 1965, Not Active, Not Active, Not Active, %s" % (mhz, cap)
+    smp.lines = [(10.00, line(1965, "Not Active")),                       # inside the 20 ms headline region
+                 (11.0, line(1500, "Active")), (11.3, line(1400, "Active")), (11.6, line(1450, "Active")),
+                 (30.0, line(300, "Not Active"))]                          # idle, outside both windows
+    head, sus = smp.stop(9.99, 10.01, 10.9, 11.9)
+    assert sus["sm_mhz"] == 1450 and sus["samples"] == 3 and sus["reasons"] == ["sw_power_cap"]
+    assert head["samples"] == 3 and "sustained leg" in head["window"]     # one sample is too few: borrowed, and said so
+    smp.proc = FakeProc()
+    head, _ = smp.stop(10.9, 11.9, 10.9, 11.9)
+    assert head["window"] == "timed region" and head["sm_max_mhz"] == 1965

@@ -6,7 +6,7 @@ import pytest
 
 import oracle
 from paper_2412_20386_b200 import workloads as wl
-from parity_util import assert_y_close, sample_row_blocks
+from parity_util import assert_y_close, row_blocks
 
 pytestmark = pytest.mark.gpu
 
@@ -25,7 +25,7 @@ def env():
     return ptq, torch
 
 
-def check_dynamic(ptq, torch, spec, B=None, full=None, x=None):
+def check_dynamic(ptq, torch, spec, B=None, x=None):
     if x is None:
         x = wl.activations(spec, wl.ROLE_EVAL, B=B)
     wq, dw, bias = wl.weights(spec)
@@ -48,9 +48,7 @@ def check_dynamic(ptq, torch, spec, B=None, full=None, x=None):
     q_ref, step_ref = oracle.quantize_dynamic(x2, s)
     assert np.array_equal(step.view(np.uint32), step_ref.view(np.uint32)), "%s: row steps differ" % spec.name
     assert np.array_equal(q, q_ref), "%s: int8 codes differ" % spec.name
-    if full is None:
-        full = M * spec.K * spec.N <= 4e9
-    blocks = [(0, M)] if full else sample_row_blocks(M, np.random.default_rng(9))
+    blocks = row_blocks(M)                       # every row, one block at a time
     for (m0, m1) in blocks:
         acc_ref = oracle.int_matmul(q_ref[m0:m1], wq)
         assert np.array_equal(acc[m0:m1], acc_ref), "%s rows %d:%d: accumulators differ" % (spec.name, m0, m1)
@@ -69,12 +67,12 @@ def test_dynamic_config0(env):
 @pytest.mark.parametrize("idx", [0, 1, 2, 3])
 def test_dynamic_config1_block_linears(env, idx):
     # K = 192, 384, 12 (generic kernel: K % 8 != 0) and 384
-    check_dynamic(*env, CFG[1][idx], full=True)
+    check_dynamic(*env, CFG[1][idx])
 
 
 @pytest.mark.parametrize("cfg,idx", [(2, 1), (3, 0), (3, 1), (4, 0)])
-def test_dynamic_large_layers_sampled(env, cfg, idx):
-    check_dynamic(*env, CFG[cfg][idx], full=False)
+def test_dynamic_large_layers_every_row(env, cfg, idx):
+    check_dynamic(*env, CFG[cfg][idx])
 
 
 def test_dynamic_special_rows(env):

@@ -31,29 +31,42 @@ def test_config0_vim_ti_out_proj_single_image(env):
     check_layer(ptq, torch, CFG[0][0])
 
 
-@pytest.mark.parametrize("idx", [0, 1, 2, 3, 4 * 23 + 0, 4 * 11 + 1, 4 * 7 + 2, 4 * 17 + 3])
+C1_ALL_PATHS = [0, 1, 2, 3, 4 * 23 + 0, 4 * 11 + 1, 4 * 7 + 2, 4 * 17 + 3]
+
+
+@pytest.mark.parametrize("idx", C1_ALL_PATHS)
 def test_config1_vim_ti_block_linears_batch64(env, idx):
     ptq, torch = env
-    clip = check_layer(ptq, torch, CFG[1][idx], full=True)
+    clip = check_layer(ptq, torch, CFG[1][idx])
     assert clip > 0      # heavy tails beyond the calibration range do clip
+
+
+@pytest.mark.parametrize("block", range(24))
+def test_config1_every_layer_default_path(env, block):
+    # all 96 linears of the 24 blocks through the default path (the eight above also take the fused and
+    # CTA-pair flags)
+    ptq, torch = env
+    for idx in range(4 * block, 4 * block + 4):
+        if idx not in C1_ALL_PATHS:
+            check_layer(ptq, torch, CFG[1][idx], flags_list=(0,))
 
 
 @pytest.mark.parametrize("idx", [0, 1])
 def test_config2_vim_s_batch128(env, idx):
     ptq, torch = env
-    check_layer(ptq, torch, CFG[2][idx], full=False)
+    check_layer(ptq, torch, CFG[2][idx])
 
 
 @pytest.mark.parametrize("idx", [0, 1])
 def test_config3_vim_b_batch256(env, idx):
     ptq, torch = env
-    check_layer(ptq, torch, CFG[3][idx], full=False)
+    check_layer(ptq, torch, CFG[3][idx])
 
 
 @pytest.mark.parametrize("idx", range(8))
 def test_config4_vmamba_stages_batch64(env, idx):
     ptq, torch = env
-    check_layer(ptq, torch, CFG[4][idx], full=False)
+    check_layer(ptq, torch, CFG[4][idx])
 
 
 def test_quantizer_all_fp16_inputs_many_scales(env):
@@ -136,7 +149,7 @@ def test_forward_edge_arguments(env):
 def test_maximum_sizes(env, K, N, T, B):
     ptq, torch = env
     spec = wl.LinearSpec(8, 1, 1, "max", B, T, K, N, bias=True, n_outliers=1)
-    check_layer(ptq, torch, spec, full=True)
+    check_layer(ptq, torch, spec)
 
 
 def test_quantizer_scales_outside_reciprocal_range_use_ieee_division(env):
@@ -177,7 +190,7 @@ def test_closed_form_integer_inputs_on_gpu(env):
 def test_odd_shapes_and_ragged_tiles(env, K, N, T, B):
     ptq, torch = env
     spec = wl.LinearSpec(9, K % 97, N % 5, "odd", B, T, K, N, bias=(N % 2 == 0))
-    check_layer(ptq, torch, spec, full=True)
+    check_layer(ptq, torch, spec)
 
 
 def test_seeded_random_shapes(env):
@@ -193,7 +206,7 @@ def test_seeded_random_shapes(env):
             K = (K + 7) // 8 * 8                     # some shapes on the vector paths
             N = (N + 7) // 8 * 8
         spec = wl.LinearSpec(8, i, i % 4, "rand%d" % i, B, T, K, N, bias=bool(i & 1))
-        check_layer(ptq, torch, spec, full=True)
+        check_layer(ptq, torch, spec)
 
 
 def test_back_to_back_layers_sharing_one_workspace(env):

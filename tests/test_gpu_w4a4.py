@@ -6,7 +6,7 @@ import pytest
 
 import oracle
 from paper_2412_20386_b200 import workloads as wl
-from parity_util import assert_y_close, sample_row_blocks
+from parity_util import assert_y_close, row_blocks
 
 pytestmark = pytest.mark.gpu
 
@@ -32,7 +32,7 @@ def weights4(spec):
     return w4, oracle.pack_int4(w4), dw, bias
 
 
-def check_w4a4(ptq, torch, spec, B=None, full=None):
+def check_w4a4(ptq, torch, spec, B=None):
     x = wl.activations(spec, wl.ROLE_EVAL, B=B)
     xcal = wl.activations(spec, wl.ROLE_CALIB)
     w4, packed, dw, bias = weights4(spec)
@@ -46,9 +46,7 @@ def check_w4a4(ptq, torch, spec, B=None, full=None):
     xd = torch.from_numpy(x).cuda()
     x2 = x.reshape(M, spec.K)
     q_ref = oracle.quantize4(x2, spec.T, s, dx)
-    if full is None:
-        full = M * spec.K * spec.N <= 4e9
-    blocks = [(0, M)] if full else sample_row_blocks(M, np.random.default_rng(3))
+    blocks = row_blocks(M)                       # every row, one block at a time
     for flags in (0, ptq.FLAG_FUSED_PROLOGUE | ptq.FLAG_CTA_PAIR):           # accepted and ignored
         y, q, acc = layer.forward_debug(xd, flags=flags)
         y2 = layer.forward(xd, flags=flags)
@@ -83,12 +81,12 @@ def test_w4a4_config0(env):
 @pytest.mark.parametrize("idx", [0, 1, 2, 3])
 def test_w4a4_config1_block_linears(env, idx):
     # K = 12 takes the generic quantize kernel; N = 44 the masked stores
-    check_w4a4(*env, CFG[1][idx], full=True)
+    check_w4a4(*env, CFG[1][idx])
 
 
 @pytest.mark.parametrize("cfg,idx", [(3, 0), (3, 1), (4, 1)])
-def test_w4a4_large_layers_sampled(env, cfg, idx):
-    check_w4a4(*env, CFG[cfg][idx], full=False)
+def test_w4a4_large_layers_every_row(env, cfg, idx):
+    check_w4a4(*env, CFG[cfg][idx])
 
 
 def test_w4a4_quantizer_all_fp16_inputs_ties_and_odd_k(env):

@@ -71,6 +71,14 @@ MUTANTS = [
      [lambda: pins.test_calibrate_degenerate_channels_and_positions()]),
     ("calibration without the floor", "if (mu < floor_) mu = floor_;", "",
      [lambda: pins.test_calibrate_degenerate_channels_and_positions()]),
+    ("per-tensor step from the raw activations", "volatile float u = ptqo_half_to_float(xcal[m * K + k]) / s[k];\n            float a = fabsf(u);\n            if (a > mu) mu = a;\n        }\n    if (mu < floor_) mu = floor_;",
+     "volatile float u = ptqo_half_to_float(xcal[m * K + k]);\n            float a = fabsf(u);\n            if (a > mu) mu = a;\n        }\n    if (mu < floor_) mu = floor_;",
+     [lambda: pins.test_calibrate_per_tensor_vs_numpy_float32_and_invariants()]),
+    ("per-tensor step over 128 levels", "volatile float d = mu / 127.0f;\n        *delta = d;", "volatile float d = mu / 128.0f;\n        *delta = d;",
+     [lambda: pins.test_calibrate_per_tensor_vs_numpy_float32_and_invariants()]),
+    ("per-tensor step of the last position only", "    for (m = 0; m < M; ++m)\n        for (k = 0; k < K; ++k) {\n            volatile float u = ptqo_half_to_float(xcal[m * K + k]) / s[k];\n            float a = fabsf(u);\n            if (a > mu) mu = a;",
+     "    for (m = T - 1; m < M; m += T)\n        for (k = 0; k < K; ++k) {\n            volatile float u = ptqo_half_to_float(xcal[m * K + k]) / s[k];\n            float a = fabsf(u);\n            if (a > mu) mu = a;",
+     [lambda: pins.test_calibrate_per_tensor_vs_numpy_float32_and_invariants()]),
     ("search: error with the wrong sign of the dequantized value", "e = fmaf(-delta, r, u);", "e = fmaf(delta, r, u);",
      [lambda: spins.test_search_zero_loss_on_grid_points_and_ties_keep_the_largest_ratio()]),
     ("search: L1 instead of L2 loss", "acc += (double)e * (double)e;", "acc += fabs((double)e);",

@@ -395,6 +395,32 @@ def test_calibrate_degenerate_channels_and_positions():
     assert dx[0] == F32(F32(1e-5) / F32(127))
 
 
+def test_calibrate_per_tensor_vs_numpy_float32_and_invariants():
+    # the per-tensor static comparator: one step for the whole tensor (latency table of Sec. 6, Fig. 5)
+    spec = wl.configs()[1][1]          # x_proj 384 -> 44
+    xcal = wl.activations(spec, wl.ROLE_CALIB)
+    wq, dw, _ = wl.weights(spec)
+    s, delta = oracle.calibrate_per_tensor(xcal, wq, dw)
+    s_np, dx_np = numpy_calibrate(xcal, wq, dw)
+    assert np.array_equal(s.view(np.uint32), s_np.view(np.uint32))
+    # independent numpy float32 evaluation of max|x/s| / 127 over the whole batch
+    u = (xcal.astype(F32) / s_np[None, None, :]).astype(F32)
+    want = F32(max(F32(np.abs(u).max()), F32(1e-5)) / F32(127))
+    assert F32(delta).view(np.uint32) == want.view(np.uint32)
+    # it is the largest of the per-position steps (division by 127 is monotonic), strictly above most of them
+    assert delta == dx_np.max() and (dx_np < delta).sum() >= spec.T - 2
+    # one step for all positions never clips the calibration batch, reaches +-127 somewhere, and wastes
+    # range at the quiet positions: that is what the per-token steps repair (Sec. 4.1 and 5.1)
+    q = oracle.quantize(xcal.reshape(-1, spec.K), spec.T, s, np.full(spec.T, delta, F32)).astype(np.int32)
+    assert q.min() >= -127 and q.max() <= 127 and np.abs(q).max() == 127
+    per_t = np.abs(q).reshape(-1, spec.T, spec.K).max(axis=(0, 2))
+    assert (per_t < 127).sum() >= spec.T - 2 and per_t[98] < 32          # the class-token row uses a fraction of the range
+    # degenerate batch: the floor
+    z = np.zeros((2, 3, 4), np.float16)
+    _, d0 = oracle.calibrate_per_tensor(z, np.ones((2, 4), np.int8), np.array([0.01, 0.02], F32))
+    assert d0 == F32(F32(1e-5) / F32(127))
+
+
 # --------------------------------------------------------------------------- #
 # input generator                                                              #
 # --------------------------------------------------------------------------- #
