@@ -91,6 +91,10 @@ ptq_status_t make_map_2d(CUtensorMap *map, CUtensorMapDataType dt, int elem_byte
     return PTQ_OK;
 }
 
+#ifndef PTQ_GEMM_SHORT_K_BLOCKS
+#define PTQ_GEMM_SHORT_K_BLOCKS 3
+#endif
+
 inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
 inline int gcd_int(int a, int b) { while (b) { int t = a % b; a = b; b = t; } return a; }
 
@@ -118,6 +122,7 @@ struct ptq_linear {
     int *d_zp = nullptr;                                 // [T] zero offsets (asymmetric layers only)
     int *d_wsum = nullptr;                               // row sums of Wq, padded like d_dw (asymmetric only)
     bool asym = false;
+    bool has_bias = false;     // false: d_bias is all zeros
     int act_bits = 8;          // 8: codes in [-128,127] (or [0,255]); 4: codes in [-8,7], one per byte
     unsigned *d_status = nullptr;
     CUtensorMap tmW;
@@ -374,6 +379,13 @@ ptq_status_t launch_gemm(const ptq_linear *h, const void *codes, long long M, vo
     p.dx = dx_rows ? dx_rows : h->d_dx;
     p.dw = h->d_dw;
     p.bias = h->d_bias;
+    p.has_bias = h->has_bias ? 1 : 0;
+    // Short main loops (up to three k-blocks per tile, K <= 384) leave the epilogue little time: three stages and two
+    // staging boxes per warp; longer ones keep four stages.  Layers with a bias hold two more scale copies.
+    const bool short_k = h->k_blocks <= PTQ_GEMM_SHORT_K_BLOCKS;
+    p.stages = (short_k || h->has_bias) ? ptq::kStages - 1 : ptq::kStages;
+    p.boxes = short_k ? 2 : 1;
+    const int gemm_smem = ptq::gemm_smem_bytes(p.stages, p.boxes, p.has_bias);
     p.y = static_cast<__half *>(y);
     p.acc_out = static_cast<int32_t *>(acc_out);
     p.status = h->d_status;
@@ -409,9 +421,9 @@ ptq_status_t launch_gemm(const ptq_linear *h, const void *codes, long long M, vo
     const long long tiles = static_cast<long long>(p.m_tiles) * p.n_tiles;
     const int grid = static_cast<int>(tiles < h->num_sms ? tiles : h->num_sms);
     if (acc_out)
-        PTQ_CUDA(launch_pdl(ptq::ptq_gemm_dequant_kernel<true>, grid, ptq::kGemmThreads, ptq::kGemmSmemBytes, stream, tmA, h->tmW, tmY, p));
+        PTQ_CUDA(launch_pdl(ptq::ptq_gemm_dequant_kernel<true>, grid, ptq::kGemmThreads, gemm_smem, stream, tmA, h->tmW, tmY, p));
     else
-        PTQ_CUDA(launch_pdl(ptq::ptq_gemm_dequant_kernel<false>, grid, ptq::kGemmThreads, ptq::kGemmSmemBytes, stream, tmA, h->tmW, tmY, p));
+        PTQ_CUDA(launch_pdl(ptq::ptq_gemm_dequant_kernel<false>, grid, ptq::kGemmThreads, gemm_smem, stream, tmA, h->tmW, tmY, p));
     g_launches.fetch_add(1, std::memory_order_relaxed);
     PTQ_CUDA(cudaGetLastError());
     return PTQ_OK;
@@ -486,6 +498,7 @@ ptq_status_t launch_fused(const ptq_linear *h, const void *x, long long M, void 
     p.dx = h->d_dx;
     p.dw = h->d_dw;
     p.bias = h->d_bias;
+    p.has_bias = h->has_bias ? 1 : 0;
     p.y = static_cast<__half *>(y);
     p.acc_out = static_cast<int32_t *>(acc_out);
     p.status = h->d_status;
@@ -651,6 +664,7 @@ static ptq_status_t create_impl(ptq_linear_t **out, int K, int N, int T, const i
     h->last_mmas = (K - (h->k_blocks - 1) * ptq::kBK + 31) / 32;
 
     h->asym = act_zero != nullptr;
+    h->has_bias = bias != nullptr;
     h->act_bits = act_bits;
     choose_astat(h);
     if (h->asym || act_bits != 8) h->as_ok = false;   // these layers run the quantize kernel + single-CTA GEMM kernel only
@@ -967,6 +981,10 @@ ptq_status_t ptq_linear_device_status(const ptq_linear_t *h)
     unsigned word = 0;
     PTQ_CUDA(cudaDeviceSynchronize());
     PTQ_CUDA(cudaMemcpy(&word, h->d_status, sizeof(word), cudaMemcpyDeviceToHost));
+    if (word & ptq::PTQ_DEV_SMEM_ALIGN) {
+        PTQ_CUDA(cudaMemset(h->d_status, 0, sizeof(word)));
+        return fail(PTQ_ERR_CUDA, "a kernel found its shared memory misaligned and did not run (status word 0x%x); its output is undefined", word);
+    }
     if (word) {
         PTQ_CUDA(cudaMemset(h->d_status, 0, sizeof(word)));
         return fail(PTQ_ERR_TIMEOUT, "a kernel abandoned a bounded wait (status word 0x%x); its output is undefined", word);

@@ -49,8 +49,23 @@ constexpr int kNumBarriers = 2 * kStages + 4;
 constexpr bool kStreamBox64 = PTQ_STORE_BOX64 != 0;
 constexpr int kStreamBoxCols = kStreamBox64 ? 64 : kStoreBoxCols;
 constexpr int kStreamStagingPerWarp = kStreamBox64 ? 32 * 128 : kStagingBytesPerWarp;
-constexpr int kGemmSmemBytes =
-    1024 + kStages * kStageBytes + kNumEpiWarps * kStreamStagingPerWarp + kNumBarriers * 8 + 16;
+// Streaming kernel: per-tile copies of the weight steps (and of the bias, for layers that have one) in
+// shared memory, double buffered by tile parity, so that the conversion loop reads them with broadcast
+// shared-memory loads instead of global loads.  Layers with a bias run three stages to make room.
+constexpr int kScaleBufBytes = kMaxBN * 4;                // one vector of one tile
+constexpr int kGemmNumBarriers = kNumBarriers + 1;        // + the barrier that publishes the scale copies
+// Two shapes of the shared memory: four stages and one staging box per epilogue warp, or three stages
+// and two boxes per warp (a step then never waits for the store before it; chosen where the main loop
+// of a tile is short, so that the epilogue is what must keep up).
+__host__ __device__ constexpr int gemm_smem_bytes(int stages, int boxes, int has_bias)
+{
+    // no slack for alignment: the dynamic shared memory array is declared 1024-byte aligned (checked at run time)
+    return stages * kStageBytes + boxes * kNumEpiWarps * kStreamStagingPerWarp + (has_bias ? 4 : 2) * kScaleBufBytes +
+           kGemmNumBarriers * 8 + 16;
+}
+constexpr int kGemmSmemBytes = gemm_smem_bytes(kStages, 1, 0);
+static_assert(kGemmSmemBytes <= 232448 && gemm_smem_bytes(kStages - 1, 2, 1) <= kGemmSmemBytes,
+              "streaming GEMM kernel exceeds the shared memory of one CTA");
 
 struct GemmParams {
     long long M;
@@ -62,6 +77,9 @@ struct GemmParams {
     const float *dx;   // [T]
     const float *dw;   // [>= n_tiles*BN + 64], zero padded
     const float *bias; // same length, zeros when the layer has no bias
+    int has_bias;      // 0: bias is all zeros and need not be read
+    int stages;        // streaming kernel: shared-memory stages (3 or 4) ...
+    int boxes;         // ... and staging boxes per epilogue warp (2 with three stages, 1 with four)
     __half *y;         // [M,N]
     int32_t *acc_out;  // [M,N] or nullptr (parity tap)
     unsigned *status;  // device status word
@@ -89,10 +107,12 @@ __device__ __forceinline__ uint32_t pack_half2(float a, float b)
     return *reinterpret_cast<uint32_t *>(&h);
 }
 
+// No "memory" clobber on purpose: the store stays ordered with the other volatile statements (the
+// fence.proxy.async and the TMA store that follow it), while ordinary loads of the scale vectors may be
+// scheduled across it, which is what keeps their latency off the conversion loop.
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint4 v)
 {
-    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
-                 : "memory");
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w));
 }
 
 // Convert 32 accumulator columns of this thread's row and write them as the four 16-byte chunks of the
@@ -272,6 +292,109 @@ __device__ __forceinline__ uint32_t epilogue_tile(const GemmParams &p, const CUt
     return nboxes;
 }
 
+// Epilogue of one 128 x BN accumulator for one warp of the streaming kernel (TMA-store path).  As
+// epilogue_tile with one 64-column box per step, except that the weight steps (and the bias) of the tile
+// are read from their copy in shared memory (`dw_s`, `bias_s`: this tile's BN floats, indexed by the
+// column inside the tile) with broadcast loads: no global-memory latency sits in the conversion loop.
+// With two staging boxes per warp (`two_boxes`) a step never waits for the store of the step before it.
+__device__ __forceinline__ uint32_t pack_half2(float2 r) { return pack_half2(r.x, r.y); }
+
+// Two accumulators at a time with the packed binary32 instructions of sm_100 (each lane of a packed
+// operation is the ordinary correctly rounded one): (float(acc) * dx) * dw + bias, then one conversion
+// of the pair to binary16.  All 64 columns are converted before the first store, which leaves the
+// instruction scheduler free to interleave the eight independent groups.
+__device__ __forceinline__ void convert_stage64_sw128(const uint32_t (&v0)[32], const uint32_t (&v1)[32], float dxr,
+                                                      const float4 *dw_s, const float4 *bias_s, uint32_t row_addr,
+                                                      int lane)
+{
+    const uint32_t sw = static_cast<uint32_t>(lane & 7);
+    const float2 dx2 = make_float2(dxr, dxr);
+    uint4 o[8];
+#pragma unroll
+    for (int jj = 0; jj < 8; ++jj) {
+        const uint32_t (&v)[32] = jj < 4 ? v0 : v1;
+        const int j8 = 8 * (jj & 3);
+        const float4 w0 = dw_s[2 * jj], w1 = dw_s[2 * jj + 1];
+        float4 b0 = make_float4(0.0f, 0.0f, 0.0f, 0.0f), b1 = b0;
+        if (bias_s != nullptr) {
+            b0 = bias_s[2 * jj];
+            b1 = bias_s[2 * jj + 1];
+        }
+        auto f = [](uint32_t a) { return __int2float_rn(static_cast<int>(a)); };
+        const float2 a0 = __fmul2_rn(make_float2(f(v[j8 + 0]), f(v[j8 + 1])), dx2);
+        const float2 a1 = __fmul2_rn(make_float2(f(v[j8 + 2]), f(v[j8 + 3])), dx2);
+        const float2 a2 = __fmul2_rn(make_float2(f(v[j8 + 4]), f(v[j8 + 5])), dx2);
+        const float2 a3 = __fmul2_rn(make_float2(f(v[j8 + 6]), f(v[j8 + 7])), dx2);
+        o[jj].x = pack_half2(__ffma2_rn(a0, make_float2(w0.x, w0.y), make_float2(b0.x, b0.y)));
+        o[jj].y = pack_half2(__ffma2_rn(a1, make_float2(w0.z, w0.w), make_float2(b0.z, b0.w)));
+        o[jj].z = pack_half2(__ffma2_rn(a2, make_float2(w1.x, w1.y), make_float2(b1.x, b1.y)));
+        o[jj].w = pack_half2(__ffma2_rn(a3, make_float2(w1.z, w1.w), make_float2(b1.z, b1.w)));
+    }
+#pragma unroll
+    for (int jj = 0; jj < 8; ++jj) st_shared_v4(row_addr + ((static_cast<uint32_t>(jj) ^ sw) << 4), o[jj]);
+}
+
+template <bool kDebugAcc>
+__device__ __forceinline__ uint32_t epilogue_tile_stream(const GemmParams &p, const CUtensorMap *tmY, uint32_t tmem_row,
+                                                         long long m_row0, int n0, float dxr, uint32_t staging,
+                                                         const float *dw_s, const float *bias_s, uint32_t nboxes,
+                                                         int lane, int col_half, int zr, bool two_boxes)
+{
+    const long long m = m_row0 + lane;
+    const bool row_ok = m < p.M;
+    for (int c0 = col_half * kEpiStepCols; c0 < p.BN; c0 += 2 * kEpiStepCols) {
+        const int n_first = n0 + c0;
+        uint32_t v0[32], v1[32];
+        tmem_ld_32x32(tmem_row + c0, v0);
+        tmem_ld_32x32(tmem_row + c0 + 32, v1);
+        tmem_ld_wait();
+        if (p.zp != nullptr) {
+            // offset-free accumulator: acc - z[t] * sum_k Wq[n,k]
+#pragma unroll
+            for (int i4 = 0; i4 < 8; ++i4) {
+                const int4 wa = __ldg(reinterpret_cast<const int4 *>(p.wsum + n_first) + i4);
+                const int4 wb = __ldg(reinterpret_cast<const int4 *>(p.wsum + n_first + 32) + i4);
+                v0[4 * i4 + 0] -= static_cast<uint32_t>(zr * wa.x);
+                v0[4 * i4 + 1] -= static_cast<uint32_t>(zr * wa.y);
+                v0[4 * i4 + 2] -= static_cast<uint32_t>(zr * wa.z);
+                v0[4 * i4 + 3] -= static_cast<uint32_t>(zr * wa.w);
+                v1[4 * i4 + 0] -= static_cast<uint32_t>(zr * wb.x);
+                v1[4 * i4 + 1] -= static_cast<uint32_t>(zr * wb.y);
+                v1[4 * i4 + 2] -= static_cast<uint32_t>(zr * wb.z);
+                v1[4 * i4 + 3] -= static_cast<uint32_t>(zr * wb.w);
+            }
+        }
+        if (kDebugAcc) {
+            if (p.acc_out != nullptr && row_ok) {
+                store_acc32(v0, p.acc_out + m * p.N, n_first, p.N);
+                store_acc32(v1, p.acc_out + m * p.N, n_first + 32, p.N);
+            }
+        }
+        // the store that last used this box must have read it before it is refilled
+        const uint32_t box = staging + ((two_boxes && (nboxes & 1u)) ? static_cast<uint32_t>(kStreamStagingPerWarp) : 0u);
+        if (lane == 0) {
+            if (two_boxes) {
+                if (nboxes >= 2u) bulk_wait_group_read<1>();
+            } else if (nboxes >= 1u) {
+                bulk_wait_group_read<0>();
+            }
+        }
+        __syncwarp();
+        convert_stage64_sw128(v0, v1, dxr, reinterpret_cast<const float4 *>(dw_s + c0),
+                              bias_s != nullptr ? reinterpret_cast<const float4 *>(bias_s + c0) : nullptr,
+                              box + static_cast<uint32_t>(lane) * 128u, lane);
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+            if (n_first < p.N && m_row0 < p.M)
+                tma_store_2d(tmY, n_first, static_cast<int>(m_row0), box);   // clipped at N and M
+            bulk_commit_group();
+        }
+        ++nboxes;
+    }
+    return nboxes;
+}
+
 // --- the kernel ---------------------------------------------------------------------------------
 
 template <bool kDebugAcc>
@@ -279,25 +402,33 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
 ptq_gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
                         const __grid_constant__ CUtensorMap tmY, const GemmParams p)
 {
-    extern __shared__ uint8_t smem_raw[];
-    const uint32_t raw = smem_u32(smem_raw);
-    const uint32_t base = (raw + 1023u) & ~1023u;                    // swizzled tiles need 1024-byte alignment
-    uint8_t *base_ptr = smem_raw + (base - raw);
-    const uint32_t staging_base = base + kStages * kStageBytes;
-    const uint32_t bar_off = kStages * kStageBytes + kNumEpiWarps * kStreamStagingPerWarp;
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    const uint32_t base = smem_u32(smem_raw);                        // swizzled tiles need 1024-byte alignment
+    if ((base & 1023u) != 0u) {
+        // never expected (the array is declared 1024-byte aligned); the layout below has no slack for it
+        if (threadIdx.x == 0) atomicOr(p.status, PTQ_DEV_SMEM_ALIGN);
+        return;
+    }
+    const uint32_t nstages = static_cast<uint32_t>(p.stages);
+    const bool two_boxes = p.boxes == 2;
+    const uint32_t staging_off = nstages * kStageBytes;
+    const uint32_t scale_off = staging_off + static_cast<uint32_t>(p.boxes) * kNumEpiWarps * kStreamStagingPerWarp;
+    const uint32_t bar_off = scale_off + (p.has_bias ? 4 : 2) * kScaleBufBytes;
+    const uint32_t staging_base = base + staging_off;
     const uint32_t bar_base = base + bar_off;
     auto full_bar = [&](uint32_t s) { return bar_base + 8u * s; };
     auto empty_bar = [&](uint32_t s) { return bar_base + 8u * (kStages + s); };
     auto tfull_bar = [&](uint32_t b) { return bar_base + 8u * (2 * kStages + b); };
     auto tempty_bar = [&](uint32_t b) { return bar_base + 8u * (2 * kStages + 2 + b); };
-    volatile uint32_t *tmem_holder = reinterpret_cast<volatile uint32_t *>(base_ptr + bar_off + kNumBarriers * 8);
+    const uint32_t scale_bar = bar_base + 8u * kNumBarriers;
+    volatile uint32_t *tmem_holder = reinterpret_cast<volatile uint32_t *>(smem_raw + bar_off + kGemmNumBarriers * 8);
     volatile uint32_t *abort_flag = tmem_holder + 1;
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
-        for (uint32_t s = 0; s < kStages; ++s) {
+        for (uint32_t s = 0; s < nstages; ++s) {
             mbar_init(full_bar(s), 1);
             mbar_init(empty_bar(s), 1);
         }
@@ -305,6 +436,7 @@ ptq_gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             mbar_init(tfull_bar(b), 1);
             mbar_init(tempty_bar(b), kNumEpiWarps);
         }
+        mbar_init(scale_bar, kNumEpiWarps);
         *abort_flag = 0u;
         fence_mbar_init();
         prefetch_tensormap(&tmA);
@@ -345,7 +477,7 @@ ptq_gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                     tma_load_2d(a_dst, &tmA, kb * kBK, m_tile * kBM, full_bar(stage));
                     tma_load_2d(a_dst + kATileBytes, &tmW, kb * kBK, n_tile * p.BN, full_bar(stage));
                     ++issued;
-                    if (++stage == kStages) {
+                    if (++stage == nstages) {
                         stage = 0;
                         phase ^= 1u;
                     }
@@ -354,8 +486,8 @@ ptq_gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             if (!ok) {
                 // Error path only: let this thread's own loads land before the CTA gives up its
                 // shared memory (bounded; each stage's last load is at most microseconds away).
-                for (uint32_t s = 0; s < kStages; ++s) {
-                    const uint32_t uses = (issued + kStages - 1u - s) / kStages;
+                for (uint32_t s = 0; s < nstages; ++s) {
+                    const uint32_t uses = (issued + nstages - 1u - s) / nstages;
                     if (uses == 0u) continue;
                     for (int i = 0; i < 200000 && !mbar_try_wait(full_bar(s), (uses - 1u) & 1u); ++i) {
                     }
@@ -385,7 +517,7 @@ ptq_gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                     for (int j = 0; j < nmma; ++j)   // 32 bytes of K per MMA: +2 in the (>>4) address field
                         mma_i8_ss(d_tmem, a_desc + 2u * j, b_desc + 2u * j, idesc, (kb | j) != 0 ? 1u : 0u);
                     mma_commit(empty_bar(stage));    // the stage is free once these MMAs have read it
-                    if (++stage == kStages) {
+                    if (++stage == nstages) {
                         stage = 0;
                         phase ^= 1u;
                     }
@@ -400,9 +532,34 @@ ptq_gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         // ------------------------------------------------------------------ epilogue warps
         const int quarter = warp & 3;                // TMEM lanes [32*quarter, 32*quarter+32)
         const int col_half = (warp - 2) >> 2;        // which of the alternating 64-column boxes
-        const uint32_t staging = staging_base + static_cast<uint32_t>(warp - 2) * kStreamStagingPerWarp;
-        uint32_t buf = 0, bphase = 0, nboxes = 0;
-        for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+        const int et = static_cast<int>(threadIdx.x) - 64;                 // 0 .. 255 among the epilogue threads
+        const uint32_t staging = staging_base + static_cast<uint32_t>(warp - 2) * static_cast<uint32_t>(p.boxes) * kStreamStagingPerWarp;
+        float *scale_s = reinterpret_cast<float *>(smem_raw + scale_off);   // [2][BN] steps, then [2][BN] bias
+        // The weight step (and bias) of one column of tile `tile`: fetched into registers one tile ahead ...
+        float dw_next = 0.0f, bias_next = 0.0f;
+        auto fetch_scales = [&](int tile) {
+            if (tile < total_tiles && et < p.BN) {
+                const int n = (tile % p.n_tiles) * p.BN + et;
+                dw_next = __ldg(p.dw + n);
+                if (p.has_bias) bias_next = __ldg(p.bias + n);
+            }
+        };
+        // ... and published in buffer `b` once every warp is done with the tile that used that buffer last
+        auto publish_scales = [&](uint32_t b) {
+            if (et < p.BN) {
+                scale_s[b * kMaxBN + et] = dw_next;
+                if (p.has_bias) scale_s[(2 + b) * kMaxBN + et] = bias_next;
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(scale_bar);
+        };
+        uint32_t buf = 0, bphase = 0, nboxes = 0, it = 0;
+        if (p.use_tma_store) {
+            fetch_scales(blockIdx.x);
+            publish_scales(0u);
+        }
+        for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++it) {
+            if (p.use_tma_store) fetch_scales(tile + static_cast<int>(gridDim.x));   // in flight during this tile
             const int m_tile = tile / p.n_tiles;
             const int n_tile = tile - m_tile * p.n_tiles;
             const long long m_row0 = static_cast<long long>(m_tile) * kBM + quarter * 32;
@@ -410,18 +567,31 @@ ptq_gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             const int t_row = (m < p.M) ? static_cast<int>(m % p.T) : 0;
             const float dxr = (m < p.M) ? __ldg(p.dx + t_row) : 0.0f;
             const int zr = (p.zp != nullptr) ? __ldg(p.zp + t_row) : 0;
-            bool got = mbar_wait(tfull_bar(buf), bphase, abort_flag, p.status);
+            bool got = true;
+            // every epilogue warp has written its share of this tile's scale copies (arrival `it` of the barrier)
+            if (p.use_tma_store) got = mbar_wait(scale_bar, it & 1u, abort_flag, p.status);
+            got = got && mbar_wait(tfull_bar(buf), bphase, abort_flag, p.status);
             got = __all_sync(0xffffffffu, got);
             if (!got) break;
             tc_fence_after_sync();
             const uint32_t tmem_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * kMaxBN;
-            nboxes = epilogue_tile<kDebugAcc, false, kStreamBox64>(p, &tmY, tmem_row, m_row0, n_tile * p.BN, dxr, staging,
-                                                                   nboxes, lane, col_half, zr);
+            if (p.use_tma_store) {
+                const float *dw_s = scale_s + (it & 1u) * kMaxBN;
+                const float *bias_s = p.has_bias ? scale_s + (2u + (it & 1u)) * kMaxBN : nullptr;
+                nboxes = epilogue_tile_stream<kDebugAcc>(p, &tmY, tmem_row, m_row0, n_tile * p.BN, dxr, staging, dw_s,
+                                                         bias_s, nboxes, lane, col_half, zr, two_boxes);
+            } else {
+                nboxes = epilogue_tile<kDebugAcc, false, kStreamBox64>(p, &tmY, tmem_row, m_row0, n_tile * p.BN, dxr,
+                                                                       staging, nboxes, lane, col_half, zr);
+            }
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(tempty_bar(buf));
             buf ^= 1u;
             if (buf == 0u) bphase ^= 1u;
+            // the next tile's scales go to the other buffer: every warp is past its reads of that buffer,
+            // because it has passed this tile's wait on scale_bar, which needed every warp's arrival
+            if (p.use_tma_store) publish_scales((it + 1u) & 1u);
         }
         if (lane == 0) bulk_wait_group<0>();         // all of this thread's stores have completed
     }

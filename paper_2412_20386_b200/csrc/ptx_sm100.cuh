@@ -13,6 +13,7 @@ namespace ptq {
 
 constexpr unsigned PTQ_DEV_OK = 0u;
 constexpr unsigned PTQ_DEV_TIMEOUT = 1u;
+constexpr unsigned PTQ_DEV_SMEM_ALIGN = 2u;   // dynamic shared memory did not start on a 1024-byte boundary
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p)
 {
