@@ -141,14 +141,22 @@ __device__ __forceinline__ float max3_abs(float a, float b, float c)
     return r;
 }
 
+// The same, but a NaN operand makes the result NaN (and keeps it NaN through a chain of these).
+__device__ __forceinline__ float max3_abs_nan(float a, float b, float c)
+{
+    float r;
+    asm("max.NaN.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(fabsf(b)), "f"(fabsf(c)));
+    return r;
+}
+
 // First-level route for signed codes, without any float-to-integer conversion instruction (those run
 // at a quarter of the rate of the other arithmetic here).  t = v' + 1.5*2^23 holds rint(v'), ties to
 // even, in its low mantissa bits, so for |v'| <= 127.25 the low BYTE of t is the two's-complement code;
 // the same t gives the tie distance.  Arithmetic is done two lanes per instruction (packed binary32
 // multiply / add / fma of sm_100; each lane is the ordinary correctly rounded operation).  Returns true
 // when the chunk has to go to the slower routes: a value within the tie band, a magnitude above
-// 127.25 (saturation is not handled here), or a NaN / infinity (their distance d is NaN, which the
-// sum below keeps while the maxima drop it).
+// 127.25 (saturation is not handled here), or a NaN / infinity: the running magnitude maximum
+// propagates NaN, and an infinity exceeds the limit, so both fail the one comparison on `big`.
 template <int kMode = kCodeS8>
 __device__ __forceinline__ bool quantize8_magic(uint32_t x0, uint32_t x1, uint32_t x2, uint32_t x3,
                                                 const float (&c8)[8], uint32_t &lo, uint32_t &hi)
@@ -156,7 +164,6 @@ __device__ __forceinline__ bool quantize8_magic(uint32_t x0, uint32_t x1, uint32
     const uint32_t xw[4] = {x0, x1, x2, x3};
     uint32_t tb[8];
     float worst = 0.0f, big = 0.0f;
-    float2 nan_acc = make_float2(0.0f, 0.0f);
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&xw[i]));
@@ -164,16 +171,14 @@ __device__ __forceinline__ bool quantize8_magic(uint32_t x0, uint32_t x1, uint32
         const float2 t = __fadd2_rn(v, make_float2(kRoundMagic, kRoundMagic));
         const float2 r = __fadd2_rn(t, make_float2(-kRoundMagic, -kRoundMagic));
         const float2 d = __ffma2_rn(v, make_float2(-1.0f, -1.0f), r);      // rint(v) - v: exact, or NaN
-        nan_acc = __fadd2_rn(nan_acc, d);
         worst = max3_abs(worst, d.x, d.y);
-        big = max3_abs(big, v.x, v.y);
+        big = max3_abs_nan(big, v.x, v.y);
         tb[2 * i] = __float_as_uint(t.x);
         tb[2 * i + 1] = __float_as_uint(t.y);
     }
     lo = pack4(static_cast<int>(tb[0]), static_cast<int>(tb[1]), static_cast<int>(tb[2]), static_cast<int>(tb[3]));
     hi = pack4(static_cast<int>(tb[4]), static_cast<int>(tb[5]), static_cast<int>(tb[6]), static_cast<int>(tb[7]));
-    const float n = __fadd_rn(nan_acc.x, nan_acc.y);
-    return !(worst <= kScreenThreshold && big <= (kMode == kCodeS4 ? 7.25f : 127.25f) && n == n);
+    return !(worst <= kScreenThreshold && big <= (kMode == kCodeS4 ? 7.25f : 127.25f));
 }
 
 // Exact route for the same 8 channels: two correctly rounded divisions per element.  s8 / rs8 point
