@@ -355,7 +355,10 @@ ptq_status_t launch_gemm(const ptq_linear *h, const void *codes, long long M, vo
     if (st != PTQ_OK) return st;
     const bool tma_store = (h->N % 8 == 0) && (reinterpret_cast<uintptr_t>(y) % 16 == 0);
     const int m_tiles_ = static_cast<int>((M + ptq::kBM - 1) / ptq::kBM);
-    const bool use_pair = want_pair && h->max_pairs > 0 &&
+#ifdef PTQ_EXP_FORCE_PAIR
+    want_pair = true;
+#endif
+    const bool use_pair = want_pair && h->max_pairs > 0 && !h->has_bias &&
                           static_cast<long long>((m_tiles_ + 1) / 2) * h->n_tiles >= h->max_pairs;
     if (tma_store) {
         st = make_map_2d(&tmY, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, y, static_cast<unsigned long long>(h->N),

@@ -622,27 +622,39 @@ ptq_gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
 constexpr int kPairStages = 6;
 constexpr int kPairBHalfBytes = (kMaxBN / 2) * kBK;                   // 16 KB
 constexpr int kPairStageBytes = kATileBytes + kPairBHalfBytes;         // 32 KB
-constexpr int kPairNumBarriers = 2 * kPairStages + 4;
-constexpr int kPairSmemBytes =
-    1024 + kPairStages * kPairStageBytes + kNumEpiWarps * kStagingBytesPerWarp + kPairNumBarriers * 8 + 16;
+constexpr int kPairNumBarriers = 2 * kPairStages + 4 + 1;              // + the barrier of the scale copies
+__host__ __device__ constexpr int pair_smem_bytes(int has_bias)
+{
+    return kPairStages * kPairStageBytes + kNumEpiWarps * kStreamStagingPerWarp + (has_bias ? 4 : 2) * kScaleBufBytes +
+           kPairNumBarriers * 8 + 16;
+}
+// layers with a bias need two more scale buffers than fit beside six stages: they take the single-CTA kernel
+constexpr int kPairSmemBytes = pair_smem_bytes(0);
+static_assert(kPairSmemBytes <= 232448, "CTA-pair GEMM kernel exceeds the shared memory of one CTA");
 
 template <bool kDebugAcc>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 ptq_gemm_dequant_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmWh,
                              const __grid_constant__ CUtensorMap tmY, const GemmParams p)
 {
-    extern __shared__ uint8_t smem_raw[];
-    const uint32_t raw = smem_u32(smem_raw);
-    const uint32_t base = (raw + 1023u) & ~1023u;
-    uint8_t *base_ptr = smem_raw + (base - raw);
-    const uint32_t staging_base = base + kPairStages * kPairStageBytes;
-    const uint32_t bar_off = kPairStages * kPairStageBytes + kNumEpiWarps * kStagingBytesPerWarp;
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    const uint32_t base = smem_u32(smem_raw);
+    const bool misaligned = (base & 1023u) != 0u;        // same in both CTAs of the pair (same kernel, same layout)
+    if (misaligned) {
+        if (threadIdx.x == 0) atomicOr(p.status, PTQ_DEV_SMEM_ALIGN);
+        return;
+    }
+    const uint32_t staging_off = kPairStages * kPairStageBytes;
+    const uint32_t scale_off = staging_off + kNumEpiWarps * kStreamStagingPerWarp;
+    const uint32_t bar_off = scale_off + 2 * kScaleBufBytes;
+    const uint32_t staging_base = base + staging_off;
     const uint32_t bar_base = base + bar_off;
     auto full_bar = [&](uint32_t s) { return bar_base + 8u * s; };
     auto empty_bar = [&](uint32_t s) { return bar_base + 8u * (kPairStages + s); };
     auto tfull_bar = [&](uint32_t b) { return bar_base + 8u * (2 * kPairStages + b); };
     auto tempty_bar = [&](uint32_t b) { return bar_base + 8u * (2 * kPairStages + 2 + b); };
-    volatile uint32_t *tmem_holder = reinterpret_cast<volatile uint32_t *>(base_ptr + bar_off + kPairNumBarriers * 8);
+    const uint32_t scale_bar = bar_base + 8u * (kPairNumBarriers - 1);
+    volatile uint32_t *tmem_holder = reinterpret_cast<volatile uint32_t *>(smem_raw + bar_off + kPairNumBarriers * 8);
     volatile uint32_t *abort_flag = tmem_holder + 1;
 
     const int warp = threadIdx.x >> 5;
@@ -661,6 +673,7 @@ ptq_gemm_dequant_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __gr
             mbar_init(tfull_bar(b), 1);
             mbar_init(tempty_bar(b), 2 * kNumEpiWarps);
         }
+        mbar_init(scale_bar, kNumEpiWarps);
         *abort_flag = 0u;
         fence_mbar_init();
         prefetch_tensormap(&tmA);
@@ -755,27 +768,51 @@ ptq_gemm_dequant_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __gr
         // ------------------------------------------------------------------ epilogue warps (both CTAs)
         const int quarter = warp & 3;
         const int col_half = (warp - 2) >> 2;
-        const uint32_t staging = staging_base + static_cast<uint32_t>(warp - 2) * kStagingBytesPerWarp;
-        uint32_t buf = 0, bphase = 0, nboxes = 0;
-        for (int tile = pair; tile < total_tiles; tile += npairs) {
+        const int et = static_cast<int>(threadIdx.x) - 64;
+        const uint32_t staging = staging_base + static_cast<uint32_t>(warp - 2) * kStreamStagingPerWarp;
+        float *scale_s = reinterpret_cast<float *>(smem_raw + scale_off);   // [2][BN] weight steps, per CTA
+        float dw_next = 0.0f;
+        auto fetch_scales = [&](int tile) {
+            if (tile < total_tiles && et < p.BN) dw_next = __ldg(p.dw + (tile % p.n_tiles) * p.BN + et);
+        };
+        auto publish_scales = [&](uint32_t b) {
+            if (et < p.BN) scale_s[b * kMaxBN + et] = dw_next;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(scale_bar);
+        };
+        uint32_t buf = 0, bphase = 0, nboxes = 0, it = 0;
+        if (p.use_tma_store) {
+            fetch_scales(pair);
+            publish_scales(0u);
+        }
+        for (int tile = pair; tile < total_tiles; tile += npairs, ++it) {
+            if (p.use_tma_store) fetch_scales(tile + npairs);
             const int m_tile = tile / p.n_tiles;
             const int n_tile = tile - m_tile * p.n_tiles;
             const long long m_row0 =
                 static_cast<long long>(m_tile) * (2 * kBM) + static_cast<long long>(rank) * kBM + quarter * 32;
             const long long m = m_row0 + lane;
             const float dxr = (m < p.M) ? __ldg(p.dx + static_cast<int>(m % p.T)) : 0.0f;
-            bool got = mbar_wait(tfull_bar(buf), bphase, abort_flag, p.status);
+            bool got = true;
+            if (p.use_tma_store) got = mbar_wait(scale_bar, it & 1u, abort_flag, p.status);
+            got = got && mbar_wait(tfull_bar(buf), bphase, abort_flag, p.status);
             got = __all_sync(0xffffffffu, got);
             if (!got) break;
             tc_fence_after_sync();
             const uint32_t tmem_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * kMaxBN;
-            nboxes = epilogue_tile<kDebugAcc, false, kStreamBox64>(p, &tmY, tmem_row, m_row0, n_tile * p.BN, dxr, staging,
-                                                                   nboxes, lane, col_half);
+            if (p.use_tma_store)
+                nboxes = epilogue_tile_stream<kDebugAcc>(p, &tmY, tmem_row, m_row0, n_tile * p.BN, dxr, staging,
+                                                         scale_s + (it & 1u) * kMaxBN, nullptr, nboxes, lane, col_half, 0,
+                                                         false);
+            else
+                nboxes = epilogue_tile<kDebugAcc, false, kStreamBox64>(p, &tmY, tmem_row, m_row0, n_tile * p.BN, dxr, staging,
+                                                                       nboxes, lane, col_half);
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive_remote(tempty_bar(buf), 0u);     // the leader's MMA thread waits on it
             buf ^= 1u;
             if (buf == 0u) bphase ^= 1u;
+            if (p.use_tma_store) publish_scales((it + 1u) & 1u);
         }
         if (lane == 0) bulk_wait_group<0>();
     }
