@@ -440,7 +440,7 @@ def run_ours(args, specs, rank, world, local_rank):
     n_each = max(3, min(args.steps, 200))
     _, step_min, step_med = event_times_ms(torch, step, n_each)
 
-    n_sus = int(min(200000, max(args.steps, SUSTAIN_SECONDS * 1e3 / max(ms_total / args.steps, 1e-4))))
+    n_sus = int(min(200000, max(args.steps, args.sustain_seconds * 1e3 / max(ms_total / args.steps, 1e-4))))
     g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     ts0 = time.time()
@@ -635,6 +635,8 @@ def main():
     ap.add_argument("--graph", action="store_true",
                     help="capture one step in a CUDA graph and time replays (for launch-bound workloads such as c1)")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--sustain-seconds", type=float, default=SUSTAIN_SECONDS,
+                    help="length of the sustained leg that follows the timed region (profiling runs shorten it)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 

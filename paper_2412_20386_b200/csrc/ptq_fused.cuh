@@ -165,8 +165,7 @@ ptq_fused_linear_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
                         const uint64_t a_desc = make_smem_desc_sw128(panel_base + kb * kATileBytes);
                         const uint64_t b_desc = make_smem_desc_sw128(w_base + stage * fp.w_stage_bytes);
                         const int nmma = (kb == p.k_blocks - 1) ? p.last_mmas : (kBK / 32);
-                        for (int j = 0; j < nmma; ++j)
-                            mma_i8_ss(d_tmem, a_desc + 2u * j, b_desc + 2u * j, idesc, (kb | j) != 0 ? 1u : 0u);
+                        mma_i8_ss_kblock(d_tmem, a_desc, b_desc, idesc, kb != 0 ? 1u : 0u, nmma);
                         mma_commit(wempty_bar(stage));
                         if (n_tile == p.n_tiles - 1) mma_commit(pempty_bar(kb));   // last reader of this panel block
                         if (++stage == static_cast<uint32_t>(fp.w_stages)) {

@@ -514,8 +514,7 @@ ptq_gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                     const uint64_t a_desc = make_smem_desc_sw128(a_addr);
                     const uint64_t b_desc = make_smem_desc_sw128(a_addr + kATileBytes);
                     const int nmma = (kb == p.k_blocks - 1) ? p.last_mmas : (kBK / 32);
-                    for (int j = 0; j < nmma; ++j)   // 32 bytes of K per MMA: +2 in the (>>4) address field
-                        mma_i8_ss(d_tmem, a_desc + 2u * j, b_desc + 2u * j, idesc, (kb | j) != 0 ? 1u : 0u);
+                    mma_i8_ss_kblock(d_tmem, a_desc, b_desc, idesc, kb != 0 ? 1u : 0u, nmma);
                     mma_commit(empty_bar(stage));    // the stage is free once these MMAs have read it
                     if (++stage == nstages) {
                         stage = 0;
@@ -750,8 +749,7 @@ ptq_gemm_dequant_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __gr
                     const uint64_t a_desc = make_smem_desc_sw128(a_addr);
                     const uint64_t b_desc = make_smem_desc_sw128(a_addr + kATileBytes);
                     const int nmma = (kb == p.k_blocks - 1) ? p.last_mmas : (kBK / 32);
-                    for (int j = 0; j < nmma; ++j)
-                        mma_i8_ss_pair(d_tmem, a_desc + 2u * j, b_desc + 2u * j, idesc, (kb | j) != 0 ? 1u : 0u);
+                    mma_i8_ss_pair_kblock(d_tmem, a_desc, b_desc, idesc, kb != 0 ? 1u : 0u, nmma);
                     mma_commit_pair(empty_bar(stage));
                     if (++stage == kPairStages) {
                         stage = 0;

@@ -213,6 +213,47 @@ __device__ __forceinline__ void mma_i8_ss(uint32_t d_tmem, uint64_t a_desc, uint
         : "memory");
 }
 
+// The four MMAs of one full k-block (128 bytes of K: the start-address field advances by 2 per 32 bytes)
+// issued back to back from ONE statement.  The tensor pipe does not queue far ahead of the issuing
+// thread: every instruction the thread spends between two MMAs (descriptor arithmetic, predicates, loop
+// control) shows up as an idle gap of the pipe, so the descriptors of all four are formed first.
+// `accumulate_first` = 0 makes the first MMA overwrite the accumulator; the other three accumulate.
+__device__ __forceinline__ void mma_i8_ss_x4(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                             uint32_t accumulate_first)
+{
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p, q;\n\t"
+        ".reg .b64 a1, a2, a3, b1, b2, b3;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "setp.eq.b32 q, 0, 0;\n\t"
+        "add.u64 a1, %1, 2;\n\t"
+        "add.u64 a2, %1, 4;\n\t"
+        "add.u64 a3, %1, 6;\n\t"
+        "add.u64 b1, %2, 2;\n\t"
+        "add.u64 b2, %2, 4;\n\t"
+        "add.u64 b3, %2, 6;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], a1, b1, %3, q;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], a2, b2, %3, q;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], a3, b3, %3, q;\n\t"
+        "}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate_first)
+        : "memory");
+}
+
+// The MMAs of one k-block: `nmma` (1..4) instructions of 32 bytes of K each.
+__device__ __forceinline__ void mma_i8_ss_kblock(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                                 uint32_t accumulate_first, int nmma)
+{
+    if (nmma == 4) {
+        mma_i8_ss_x4(d_tmem, a_desc, b_desc, idesc, accumulate_first);
+    } else {
+        for (int j = 0; j < nmma; ++j)
+            mma_i8_ss(d_tmem, a_desc + 2u * j, b_desc + 2u * j, idesc, j != 0 ? 1u : accumulate_first);
+    }
+}
+
 // mbarrier arrives once all tcgen05 operations issued so far by this thread have completed.
 __device__ __forceinline__ void mma_commit(uint32_t bar)
 {
@@ -310,6 +351,36 @@ __device__ __forceinline__ void mma_i8_ss_pair(uint32_t d_tmem, uint64_t a_desc,
         "}"
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
+}
+
+// The four MMAs of one full k-block over both CTAs of the pair, issued back to back (see mma_i8_ss_x4).
+__device__ __forceinline__ void mma_i8_ss_pair_kblock(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                                      uint32_t accumulate_first, int nmma)
+{
+    if (nmma == 4) {
+        asm volatile(
+            "{\n\t"
+            ".reg .pred p, q;\n\t"
+            ".reg .b64 a1, a2, a3, b1, b2, b3;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "setp.eq.b32 q, 0, 0;\n\t"
+            "add.u64 a1, %1, 2;\n\t"
+            "add.u64 a2, %1, 4;\n\t"
+            "add.u64 a3, %1, 6;\n\t"
+            "add.u64 b1, %2, 2;\n\t"
+            "add.u64 b2, %2, 4;\n\t"
+            "add.u64 b3, %2, 6;\n\t"
+            "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n\t"
+            "tcgen05.mma.cta_group::2.kind::i8 [%0], a1, b1, %3, q;\n\t"
+            "tcgen05.mma.cta_group::2.kind::i8 [%0], a2, b2, %3, q;\n\t"
+            "tcgen05.mma.cta_group::2.kind::i8 [%0], a3, b3, %3, q;\n\t"
+            "}"
+            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate_first)
+            : "memory");
+    } else {
+        for (int j = 0; j < nmma; ++j)
+            mma_i8_ss_pair(d_tmem, a_desc + 2u * j, b_desc + 2u * j, idesc, j != 0 ? 1u : accumulate_first);
+    }
 }
 
 // The mbarriers at this offset in both CTAs of the pair (mask 0b11) arrive once all tcgen05 operations
