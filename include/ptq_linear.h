@@ -63,7 +63,7 @@ typedef enum {
 /* Flags for create / forward. */
 #define PTQ_FLAG_NONE            0u
 #define PTQ_FLAG_FUSED_PROLOGUE  1u   /* F1: quantize inside the GEMM kernel; no int8 round trip, no workspace
-                                         (same bits; at present slower than the two-kernel path) */
+                                         (same bits; measured 2-3x slower than the two-kernel path) */
 #define PTQ_FLAG_CTA_PAIR        2u   /* two-kernel path: run G1+E1 on CTA pairs (tcgen05 cta_group::2, 256-row tiles,
                                          half the weight bytes per CTA) when the batch has enough rows; same results */
 
@@ -113,7 +113,10 @@ void ptq_linear_destroy(ptq_linear_t *h);
 /*
  * Bytes of device workspace ptq_linear_forward needs for a batch of B images:
  * the int8 codes [B*T, Kpad] with Kpad = K rounded up to 16, or 0 with
- * PTQ_FLAG_FUSED_PROLOGUE.  Returns 0 for a NULL handle or B < 1.
+ * PTQ_FLAG_FUSED_PROLOGUE on a layer the fused kernel covers.  The answer assumes a
+ * 16-byte aligned x: an x that is only 2-byte aligned always takes the two-kernel path
+ * and needs the size reported for PTQ_FLAG_NONE, whatever the flags.
+ * Returns 0 for a NULL handle or B < 1.
  */
 size_t ptq_linear_workspace_bytes(const ptq_linear_t *h, int B, unsigned flags);
 
@@ -183,7 +186,8 @@ ptq_status_t ptq_linear_forward_dynamic_debug(const ptq_linear_t *h, const void 
                                               void *q_int8_out, void *acc_int32_out, void *step_fp32_out,
                                               void *workspace, size_t workspace_bytes, void *stream);
 
-/* 1 if PTQ_FLAG_FUSED_PROLOGUE runs the single fused kernel for this layer, 0 if it falls back. */
+/* 1 if PTQ_FLAG_FUSED_PROLOGUE runs the single fused kernel for this layer (given a 16-byte aligned x;
+ * any other x falls back to the two-kernel path and needs the workspace), 0 if the layer always falls back. */
 int ptq_linear_fused_supported(const ptq_linear_t *h);
 
 /*

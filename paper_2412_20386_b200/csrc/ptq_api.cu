@@ -160,13 +160,12 @@ template <auto kKern>
 ptq_status_t ensure_smem(int device, int bytes)
 {
     constexpr int kMaxDevices = 64;
-    static std::mutex mu;
-    static bool done[kMaxDevices] = {};
+    static std::atomic<bool> done[kMaxDevices] = {};
     if (device < 0 || device >= kMaxDevices) return fail(PTQ_ERR_CUDA, "device index %d out of range", device);
-    std::lock_guard<std::mutex> lock(mu);
-    if (!done[device]) {
+    // lock-free once the attribute is set; two threads racing on the first call both set the same value
+    if (!done[device].load(std::memory_order_acquire)) {
         PTQ_CUDA(cudaFuncSetAttribute(kKern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
-        done[device] = true;
+        done[device].store(true, std::memory_order_release);
     }
     return PTQ_OK;
 }
