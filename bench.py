@@ -610,10 +610,10 @@ def run_ours(args, specs, rank, world, local_rank):
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised
 # under profiles/; keyed by (kernel, workload, layer).  An entry is removed when its kernel changes.
 TRAFFIC = {
-    ("ptq_gemm_dequant_kernel", "c3", "in_proj"): 41.173760e6 + 251.041792e6,
-    ("ptq_gemm_dequant_kernel", "c3", "out_proj"): 78.697728e6 + 31.951104e6,
-    ("ptq_quantize_kernel", "c3", "in_proj"): 77.508096e6 + 10.753792e6,
-    ("ptq_quantize_kernel", "c3", "out_proj"): 155.139072e6 + 47.510784e6,
+    ("ptq_gemm_dequant_kernel", "c3", "in_proj"): 41.165312e6 + 251.771648e6,
+    ("ptq_gemm_dequant_kernel", "c3", "out_proj"): 78.706688e6 + 33.521664e6,
+    ("ptq_quantize_kernel", "c3", "in_proj"): 77.504000e6 + 10.326528e6,
+    ("ptq_quantize_kernel", "c3", "out_proj"): 155.117824e6 + 45.882624e6,
 }
 
 
