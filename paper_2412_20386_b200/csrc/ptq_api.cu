@@ -338,6 +338,44 @@ ptq_status_t launch_quantize_dynamic(const ptq_linear *h, const void *x, long lo
     return PTQ_OK;
 }
 
+#ifndef PTQ_GEMM_PANEL
+#define PTQ_GEMM_PANEL 1
+#endif
+
+// Whether this launch takes the panel kernel (the codes of a row panel resident in shared memory for a
+// group of N tiles), and with which tiling: fills p.group, p.groups, p.b_stages, p.b_stage_bytes.
+// It pays on large compute-bound layers only (measured: 2-3 % of the Vim-B step, nothing or a loss on
+// layers with K <= 384 or few tiles), so it is taken when the layer has at least four k-blocks and
+// eight tiles per SM, and only with a group size G whose work units divide over the CTAs as evenly as
+// single tiles do: rounds(G) * G <= rounds(1).  Among those the largest G wins (fewest panel loads).
+bool plan_panel(const ptq_linear *h, ptq::GemmParams &p, bool tma_store)
+{
+    p.group = p.groups = p.b_stages = p.b_stage_bytes = 0;
+    const long long tiles = static_cast<long long>(p.m_tiles) * p.n_tiles;
+    if (!PTQ_GEMM_PANEL || !tma_store || p.n_tiles < 2 || p.k_blocks < 4 || p.k_blocks > ptq::kPanelMaxKBlocks ||
+        tiles < 8ll * h->num_sms)
+        return false;
+    const int stage_bytes = p.BN * ptq::kBK;
+    const int fixed = ptq::panel_smem_bytes(p.k_blocks, 0, 0, p.boxes, p.has_bias);
+    int stages = (ptq::kPanelSmemLimit - fixed) / stage_bytes;
+    if (stages < 3) return false;
+    if (stages > ptq::kPanelMaxBStages) stages = ptq::kPanelMaxBStages;
+    const long long rounds1 = (tiles + h->num_sms - 1) / h->num_sms;
+    int best_g = 1;
+    for (int g = 2; g <= p.n_tiles; ++g) {
+        const long long units = static_cast<long long>((p.n_tiles + g - 1) / g) * p.m_tiles;
+        const long long grid = units < h->num_sms ? units : h->num_sms;
+        const long long rounds = (units + grid - 1) / grid;
+        if (rounds * g <= rounds1) best_g = g;
+    }
+    if (best_g < 2) return false;
+    p.group = best_g;
+    p.groups = (p.n_tiles + best_g - 1) / best_g;
+    p.b_stages = stages;
+    p.b_stage_bytes = stage_bytes;
+    return true;
+}
+
 // G1+E1 launch on codes [M, Kpad] at `codes`.
 // dx_rows != nullptr: the steps are per ROW (dynamic comparator), i.e. dx = dx_rows and T = M.
 ptq_status_t launch_gemm(const ptq_linear *h, const void *codes, long long M, void *y, void *acc_out,
@@ -421,6 +459,22 @@ ptq_status_t launch_gemm(const ptq_linear *h, const void *codes, long long M, vo
         return PTQ_OK;
     }
     const long long tiles = static_cast<long long>(p.m_tiles) * p.n_tiles;
+    if (plan_panel(h, p, tma_store)) {
+        // several N tiles and K <= 768: the codes of a row panel stay in shared memory for `group` tiles
+        const int psmem = ptq::panel_smem_bytes(p.k_blocks, p.b_stages, p.b_stage_bytes, p.boxes, p.has_bias);
+        const long long units = static_cast<long long>(p.m_tiles) * p.groups;
+        const int pgrid = static_cast<int>(units < h->num_sms ? units : h->num_sms);
+        ptq_status_t ps = acc_out ? ensure_smem<ptq::ptq_gemm_dequant_panel_kernel<true>>(h->device, ptq::kPanelSmemLimit)
+                                  : ensure_smem<ptq::ptq_gemm_dequant_panel_kernel<false>>(h->device, ptq::kPanelSmemLimit);
+        if (ps != PTQ_OK) return ps;
+        if (acc_out)
+            PTQ_CUDA(launch_pdl(ptq::ptq_gemm_dequant_panel_kernel<true>, pgrid, ptq::kGemmThreads, psmem, stream, tmA, h->tmW, tmY, p));
+        else
+            PTQ_CUDA(launch_pdl(ptq::ptq_gemm_dequant_panel_kernel<false>, pgrid, ptq::kGemmThreads, psmem, stream, tmA, h->tmW, tmY, p));
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+        PTQ_CUDA(cudaGetLastError());
+        return PTQ_OK;
+    }
     const int grid = static_cast<int>(tiles < h->num_sms ? tiles : h->num_sms);
     if (acc_out)
         PTQ_CUDA(launch_pdl(ptq::ptq_gemm_dequant_kernel<true>, grid, ptq::kGemmThreads, gemm_smem, stream, tmA, h->tmW, tmY, p));

@@ -91,6 +91,10 @@ struct GemmParams {
     // accumulator sum_k (c - z[t]) * Wq[n,k] exactly (all int32).  nullptr for symmetric layers.
     const int *zp;     // [T]
     const int *wsum;   // [>= n_tiles*BN + 64] row sums of Wq, zero padded
+    // Panel kernel only: a work unit is one 128-row panel of codes times `group` adjacent N tiles; `groups`
+    // units cover a panel; the weight ring has `b_stages` slots of `b_stage_bytes` (= BN * 128) each.
+    int group, groups;
+    int b_stages, b_stage_bytes;
 };
 
 // --- epilogue helpers -------------------------------------------------------------------------
@@ -591,6 +595,274 @@ ptq_gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             // the next tile's scales go to the other buffer: every warp is past its reads of that buffer,
             // because it has passed this tile's wait on scale_bar, which needed every warp's arrival
             if (p.use_tma_store) publish_scales((it + 1u) & 1u);
+        }
+        if (lane == 0) bulk_wait_group<0>();         // all of this thread's stores have completed
+    }
+
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+// --- panel variant: the codes of a row panel stay in shared memory ------------------------------
+//
+// Same computation as the streaming kernel for layers with several N tiles and K <= 768.  A work unit
+// is one 128-row panel of codes (all its k-blocks, k_blocks x 16 KB, loaded once) times `group`
+// adjacent N tiles; only the weight tiles stream through a ring of stages.  Per output tile a CTA then
+// fetches BN x K bytes instead of (128 + BN) x K: a third less operand traffic between L2 and the SMs,
+// which is what the streaming kernel's MMA thread waits on (and what costs energy under the power
+// cap).  `group` is chosen by the host so that the units divide evenly over the CTAs; the units of one
+// panel go to neighbouring CTAs, which read the panel from L2 at about the same time.
+//
+// Barriers: afull/aempty per panel k-block (one phase per unit: the MMA thread frees k-block kb with a
+// commit after the unit's LAST tile has read it, so the next unit's panel arrives k-block by k-block
+// while that tile still runs), bfull/bempty per weight stage, tfull/tempty per accumulator, one for
+// the scale copies.  The producer interleaves the panel loads with the first tile's weight loads so
+// that a wait for a late panel slot never holds back weights whose stage is free.
+constexpr int kPanelMaxKBlocks = 6;                       // panel of at most 96 KB (K <= 768)
+constexpr int kPanelMaxBStages = 6;
+constexpr int kPanelNumBarriers = 2 * kPanelMaxKBlocks + 2 * kPanelMaxBStages + 4 + 1;
+constexpr int kPanelSmemLimit = 232448;                   // 227 KB opt-in maximum per CTA
+__host__ __device__ constexpr int panel_smem_bytes(int k_blocks, int b_stages, int b_stage_bytes, int boxes, int has_bias)
+{
+    return k_blocks * kATileBytes + b_stages * b_stage_bytes + boxes * kNumEpiWarps * kStreamStagingPerWarp +
+           (has_bias ? 4 : 2) * kScaleBufBytes + kPanelNumBarriers * 8 + 16;
+}
+
+template <bool kDebugAcc>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+ptq_gemm_dequant_panel_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
+                              const __grid_constant__ CUtensorMap tmY, const GemmParams p)
+{
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    const uint32_t base = smem_u32(smem_raw);
+    if ((base & 1023u) != 0u) {
+        if (threadIdx.x == 0) atomicOr(p.status, PTQ_DEV_SMEM_ALIGN);
+        return;
+    }
+    const uint32_t nb = static_cast<uint32_t>(p.b_stages);
+    const uint32_t b_bytes = static_cast<uint32_t>(p.b_stage_bytes);
+    const bool two_boxes = p.boxes == 2;
+    const uint32_t b_off = static_cast<uint32_t>(p.k_blocks) * kATileBytes;
+    const uint32_t staging_off = b_off + nb * b_bytes;
+    const uint32_t scale_off = staging_off + static_cast<uint32_t>(p.boxes) * kNumEpiWarps * kStreamStagingPerWarp;
+    const uint32_t bar_off = scale_off + (p.has_bias ? 4 : 2) * kScaleBufBytes;
+    const uint32_t bar_base = base + bar_off;
+    auto afull_bar = [&](uint32_t kb) { return bar_base + 8u * kb; };
+    auto aempty_bar = [&](uint32_t kb) { return bar_base + 8u * (kPanelMaxKBlocks + kb); };
+    auto bfull_bar = [&](uint32_t s) { return bar_base + 8u * (2 * kPanelMaxKBlocks + s); };
+    auto bempty_bar = [&](uint32_t s) { return bar_base + 8u * (2 * kPanelMaxKBlocks + kPanelMaxBStages + s); };
+    auto tfull_bar = [&](uint32_t b) { return bar_base + 8u * (2 * kPanelMaxKBlocks + 2 * kPanelMaxBStages + b); };
+    auto tempty_bar = [&](uint32_t b) { return bar_base + 8u * (2 * kPanelMaxKBlocks + 2 * kPanelMaxBStages + 2 + b); };
+    const uint32_t scale_bar = bar_base + 8u * (kPanelNumBarriers - 1);
+    volatile uint32_t *tmem_holder = reinterpret_cast<volatile uint32_t *>(smem_raw + bar_off + kPanelNumBarriers * 8);
+    volatile uint32_t *abort_flag = tmem_holder + 1;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (uint32_t kb = 0; kb < static_cast<uint32_t>(p.k_blocks); ++kb) {
+            mbar_init(afull_bar(kb), 1);
+            mbar_init(aempty_bar(kb), 1);
+        }
+        for (uint32_t s = 0; s < nb; ++s) {
+            mbar_init(bfull_bar(s), 1);
+            mbar_init(bempty_bar(s), 1);
+        }
+        for (uint32_t b = 0; b < 2; ++b) {
+            mbar_init(tfull_bar(b), 1);
+            mbar_init(tempty_bar(b), kNumEpiWarps);
+        }
+        mbar_init(scale_bar, kNumEpiWarps);
+        *abort_flag = 0u;
+        fence_mbar_init();
+        prefetch_tensormap(&tmA);
+        prefetch_tensormap(&tmW);
+        prefetch_tensormap(&tmY);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(const_cast<uint32_t *>(tmem_holder)), kTmemCols);
+        tmem_relinquish_alloc_permit();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_holder;
+
+    // From here on the codes (and, for the dynamic comparator, the row steps) of the kernel before are read.
+    griddep_wait();
+    griddep_launch_dependents();
+
+    const int units = p.m_tiles * p.groups;
+    // unit u -> panel u / groups, N tiles [first, first + count)
+    auto unit_first = [&](int u) { return (u % p.groups) * p.group; };
+    auto unit_count = [&](int u) {
+        const int left = p.n_tiles - unit_first(u);
+        return left < p.group ? left : p.group;
+    };
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t stage = 0, sphase = 0, uph = 0, b_issued = 0, a_units = 0;
+            int a_kb_issued = 0;                 // panel k-blocks issued for the unit in progress
+            bool ok = true;
+            for (int unit = blockIdx.x; unit < units && ok; unit += gridDim.x, uph ^= 1u) {
+                const int m_tile = unit / p.groups;
+                const int n_first = unit_first(unit), n_count = unit_count(unit);
+                a_kb_issued = 0;
+                for (int j = 0; j < n_count && ok; ++j) {
+                    for (int kb = 0; kb < p.k_blocks; ++kb) {
+                        if (j == 0) {
+                            // slot kb of the panel: free once the previous unit's last tile has read it
+                            if (!mbar_wait(aempty_bar(kb), uph ^ 1u, abort_flag, p.status)) {
+                                ok = false;
+                                break;
+                            }
+                            mbar_arrive_expect_tx(afull_bar(kb), static_cast<uint32_t>(kATileBytes));
+                            tma_load_2d(base + static_cast<uint32_t>(kb) * kATileBytes, &tmA, kb * kBK, m_tile * kBM,
+                                        afull_bar(kb));
+                            ++a_kb_issued;
+                        }
+                        if (!mbar_wait(bempty_bar(stage), sphase ^ 1u, abort_flag, p.status)) {
+                            ok = false;
+                            break;
+                        }
+                        mbar_arrive_expect_tx(bfull_bar(stage), b_bytes);
+                        tma_load_2d(base + b_off + stage * b_bytes, &tmW, kb * kBK, (n_first + j) * p.BN, bfull_bar(stage));
+                        ++b_issued;
+                        if (++stage == nb) {
+                            stage = 0;
+                            sphase ^= 1u;
+                        }
+                    }
+                }
+                if (ok) ++a_units;
+            }
+            if (!ok) {
+                // Error path only: let this thread's own loads land before the CTA gives up its shared memory (bounded).
+                for (uint32_t s = 0; s < nb; ++s) {
+                    const uint32_t uses = (b_issued + nb - 1u - s) / nb;
+                    if (uses == 0u) continue;
+                    for (int i = 0; i < 200000 && !mbar_try_wait(bfull_bar(s), (uses - 1u) & 1u); ++i) {
+                    }
+                }
+                for (int kb = 0; kb < p.k_blocks; ++kb) {
+                    const uint32_t uses = a_units + (kb < a_kb_issued ? 1u : 0u);
+                    if (uses == 0u) continue;
+                    for (int i = 0; i < 200000 && !mbar_try_wait(afull_bar(kb), (uses - 1u) & 1u); ++i) {
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = make_idesc_s8(kBM, p.BN, p.zp != nullptr);
+            uint32_t stage = 0, sphase = 0, uph = 0, buf = 0, bphase = 0;
+            bool ok = true;
+            for (int unit = blockIdx.x; unit < units && ok; unit += gridDim.x, uph ^= 1u) {
+                const int n_count = unit_count(unit);
+                for (int j = 0; j < n_count && ok; ++j) {
+                    if (!mbar_wait(tempty_bar(buf), bphase ^ 1u, abort_flag, p.status)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after_sync();
+                    const uint32_t d_tmem = tmem_base + buf * kMaxBN;
+                    for (int kb = 0; kb < p.k_blocks; ++kb) {
+                        if (j == 0 && !mbar_wait(afull_bar(kb), uph, abort_flag, p.status)) {
+                            ok = false;
+                            break;
+                        }
+                        if (!mbar_wait(bfull_bar(stage), sphase, abort_flag, p.status)) {
+                            ok = false;
+                            break;
+                        }
+                        tc_fence_after_sync();
+                        const uint64_t a_desc = make_smem_desc_sw128(base + static_cast<uint32_t>(kb) * kATileBytes);
+                        const uint64_t b_desc = make_smem_desc_sw128(base + b_off + stage * b_bytes);
+                        const int nmma = (kb == p.k_blocks - 1) ? p.last_mmas : (kBK / 32);
+                        mma_i8_ss_kblock(d_tmem, a_desc, b_desc, idesc, kb != 0 ? 1u : 0u, nmma);
+                        mma_commit(bempty_bar(stage));                       // the weight stage is free once these MMAs have read it
+                        if (j == n_count - 1) mma_commit(aempty_bar(kb));    // and, after the unit's last tile, so is the panel slot
+                        if (++stage == nb) {
+                            stage = 0;
+                            sphase ^= 1u;
+                        }
+                    }
+                    if (!ok) break;
+                    mma_commit(tfull_bar(buf));          // accumulator complete
+                    buf ^= 1u;
+                    if (buf == 0u) bphase ^= 1u;
+                }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue warps
+        const int quarter = warp & 3;
+        const int col_half = (warp - 2) >> 2;
+        const int et = static_cast<int>(threadIdx.x) - 64;
+        const uint32_t staging = base + staging_off + static_cast<uint32_t>(warp - 2) * static_cast<uint32_t>(p.boxes) * kStreamStagingPerWarp;
+        float *scale_s = reinterpret_cast<float *>(smem_raw + scale_off);   // [2][BN] steps, then [2][BN] bias
+        float dw_next = 0.0f, bias_next = 0.0f;
+        auto fetch_scales = [&](int n_tile) {
+            if (et < p.BN) {
+                const int n = n_tile * p.BN + et;
+                dw_next = __ldg(p.dw + n);
+                if (p.has_bias) bias_next = __ldg(p.bias + n);
+            }
+        };
+        auto publish_scales = [&](uint32_t b) {
+            if (et < p.BN) {
+                scale_s[b * kMaxBN + et] = dw_next;
+                if (p.has_bias) scale_s[(2 + b) * kMaxBN + et] = bias_next;
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(scale_bar);
+        };
+        uint32_t buf = 0, bphase = 0, nboxes = 0, it = 0;
+        int unit = blockIdx.x, j = 0;
+        if (unit < units) fetch_scales(unit_first(unit));
+        publish_scales(0u);
+        while (unit < units) {
+            // the tile after this one: its scales are fetched now and stay in flight during this tile
+            int next_unit = unit, next_j = j + 1;
+            if (next_j == unit_count(unit)) {
+                next_unit = unit + static_cast<int>(gridDim.x);
+                next_j = 0;
+            }
+            if (next_unit < units) fetch_scales(unit_first(next_unit) + next_j);
+            const int m_tile = unit / p.groups;
+            const int n_tile = unit_first(unit) + j;
+            const long long m_row0 = static_cast<long long>(m_tile) * kBM + quarter * 32;
+            const long long m = m_row0 + lane;
+            const int t_row = (m < p.M) ? static_cast<int>(m % p.T) : 0;
+            const float dxr = (m < p.M) ? __ldg(p.dx + t_row) : 0.0f;
+            const int zr = (p.zp != nullptr) ? __ldg(p.zp + t_row) : 0;
+            bool got = mbar_wait(scale_bar, it & 1u, abort_flag, p.status);
+            got = got && mbar_wait(tfull_bar(buf), bphase, abort_flag, p.status);
+            got = __all_sync(0xffffffffu, got);
+            if (!got) break;
+            tc_fence_after_sync();
+            const uint32_t tmem_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * kMaxBN;
+            const float *dw_s = scale_s + (it & 1u) * kMaxBN;
+            const float *bias_s = p.has_bias ? scale_s + (2u + (it & 1u)) * kMaxBN : nullptr;
+            nboxes = epilogue_tile_stream<kDebugAcc>(p, &tmY, tmem_row, m_row0, n_tile * p.BN, dxr, staging, dw_s, bias_s,
+                                                     nboxes, lane, col_half, zr, two_boxes);
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty_bar(buf));
+            buf ^= 1u;
+            if (buf == 0u) bphase ^= 1u;
+            publish_scales((it + 1u) & 1u);
+            unit = next_unit;
+            j = next_j;
+            ++it;
         }
         if (lane == 0) bulk_wait_group<0>();         // all of this thread's stores have completed
     }
