@@ -341,6 +341,12 @@ ptq_status_t launch_quantize_dynamic(const ptq_linear *h, const void *x, long lo
 #ifndef PTQ_GEMM_PANEL
 #define PTQ_GEMM_PANEL 1
 #endif
+#ifndef PTQ_GEMM_TEAMS
+#define PTQ_GEMM_TEAMS 1
+#endif
+#ifndef PTQ_GEMM_TEAM_MIN_ROUNDS
+#define PTQ_GEMM_TEAM_MIN_ROUNDS 4
+#endif
 
 // Whether this launch takes the panel kernel (the codes of a row panel resident in shared memory for a
 // group of N tiles), and with which tiling: fills p.group, p.groups, p.b_stages, p.b_stage_bytes.
@@ -381,10 +387,6 @@ bool plan_panel(const ptq_linear *h, ptq::GemmParams &p, bool tma_store)
 ptq_status_t launch_gemm(const ptq_linear *h, const void *codes, long long M, void *y, void *acc_out,
                          cudaStream_t stream, bool want_pair = false, const float *dx_rows = nullptr)
 {
-    ptq_status_t attr_status = ensure_smem<ptq::ptq_gemm_dequant_kernel<false>>(h->device, ptq::kGemmSmemBytes);
-    if (attr_status == PTQ_OK) attr_status = ensure_smem<ptq::ptq_gemm_dequant_kernel<true>>(h->device, ptq::kGemmSmemBytes);
-    if (attr_status != PTQ_OK) return attr_status;
-
     CUtensorMap tmA, tmY;
     ptq_status_t st = make_map_2d(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, codes, static_cast<unsigned long long>(h->K),
                                   static_cast<unsigned long long>(M), static_cast<unsigned long long>(h->Kpad),
@@ -459,15 +461,20 @@ ptq_status_t launch_gemm(const ptq_linear *h, const void *codes, long long M, vo
         return PTQ_OK;
     }
     const long long tiles = static_cast<long long>(p.m_tiles) * p.n_tiles;
+    // Short main loop (K <= 384) and several tiles per CTA: the epilogue sets the pace and runs in two teams of
+    // four warps, one per accumulator; otherwise all eight warps share every tile (shorter latency of a tile).
+    const bool teams = PTQ_GEMM_TEAMS && tma_store && short_k &&
+                       tiles >= static_cast<long long>(PTQ_GEMM_TEAM_MIN_ROUNDS) * h->num_sms;
+    const bool dbg = acc_out != nullptr;
     if (plan_panel(h, p, tma_store)) {
-        // several N tiles and K <= 768: the codes of a row panel stay in shared memory for `group` tiles
+        // several N tiles and 512 <= K <= 768: the codes of a row panel stay in shared memory for `group` tiles
         const int psmem = ptq::panel_smem_bytes(p.k_blocks, p.b_stages, p.b_stage_bytes, p.boxes, p.has_bias);
         const long long units = static_cast<long long>(p.m_tiles) * p.groups;
         const int pgrid = static_cast<int>(units < h->num_sms ? units : h->num_sms);
-        ptq_status_t ps = acc_out ? ensure_smem<ptq::ptq_gemm_dequant_panel_kernel<true>>(h->device, ptq::kPanelSmemLimit)
-                                  : ensure_smem<ptq::ptq_gemm_dequant_panel_kernel<false>>(h->device, ptq::kPanelSmemLimit);
+        ptq_status_t ps = dbg ? ensure_smem<ptq::ptq_gemm_dequant_panel_kernel<true>>(h->device, ptq::kPanelSmemLimit)
+                              : ensure_smem<ptq::ptq_gemm_dequant_panel_kernel<false>>(h->device, ptq::kPanelSmemLimit);
         if (ps != PTQ_OK) return ps;
-        if (acc_out)
+        if (dbg)
             PTQ_CUDA(launch_pdl(ptq::ptq_gemm_dequant_panel_kernel<true>, pgrid, ptq::kGemmThreads, psmem, stream, tmA, h->tmW, tmY, p));
         else
             PTQ_CUDA(launch_pdl(ptq::ptq_gemm_dequant_panel_kernel<false>, pgrid, ptq::kGemmThreads, psmem, stream, tmA, h->tmW, tmY, p));
@@ -476,10 +483,21 @@ ptq_status_t launch_gemm(const ptq_linear *h, const void *codes, long long M, vo
         return PTQ_OK;
     }
     const int grid = static_cast<int>(tiles < h->num_sms ? tiles : h->num_sms);
-    if (acc_out)
-        PTQ_CUDA(launch_pdl(ptq::ptq_gemm_dequant_kernel<true>, grid, ptq::kGemmThreads, gemm_smem, stream, tmA, h->tmW, tmY, p));
-    else
-        PTQ_CUDA(launch_pdl(ptq::ptq_gemm_dequant_kernel<false>, grid, ptq::kGemmThreads, gemm_smem, stream, tmA, h->tmW, tmY, p));
+    auto go = [&](auto kern) -> ptq_status_t {
+        PTQ_CUDA(launch_pdl(kern, grid, ptq::kGemmThreads, gemm_smem, stream, tmA, h->tmW, tmY, p));
+        return PTQ_OK;
+    };
+    ptq_status_t gs;
+    if (teams) {
+        gs = dbg ? ensure_smem<ptq::ptq_gemm_dequant_kernel<true, true>>(h->device, ptq::kGemmSmemBytes)
+                 : ensure_smem<ptq::ptq_gemm_dequant_kernel<false, true>>(h->device, ptq::kGemmSmemBytes);
+        if (gs == PTQ_OK) gs = dbg ? go(ptq::ptq_gemm_dequant_kernel<true, true>) : go(ptq::ptq_gemm_dequant_kernel<false, true>);
+    } else {
+        gs = dbg ? ensure_smem<ptq::ptq_gemm_dequant_kernel<true, false>>(h->device, ptq::kGemmSmemBytes)
+                 : ensure_smem<ptq::ptq_gemm_dequant_kernel<false, false>>(h->device, ptq::kGemmSmemBytes);
+        if (gs == PTQ_OK) gs = dbg ? go(ptq::ptq_gemm_dequant_kernel<true, false>) : go(ptq::ptq_gemm_dequant_kernel<false, false>);
+    }
+    if (gs != PTQ_OK) return gs;
     g_launches.fetch_add(1, std::memory_order_relaxed);
     PTQ_CUDA(cudaGetLastError());
     return PTQ_OK;

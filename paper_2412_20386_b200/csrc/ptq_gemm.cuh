@@ -296,7 +296,8 @@ __device__ __forceinline__ uint32_t epilogue_tile(const GemmParams &p, const CUt
     return nboxes;
 }
 
-// Epilogue of one 128 x BN accumulator for one warp of the streaming kernel (TMA-store path).  As
+// Epilogue of one 128 x BN accumulator for one warp of the streaming kernel (TMA-store path); the warp
+// takes the 64-column steps c_begin, c_begin + c_stride, ...  As
 // epilogue_tile with one 64-column box per step, except that the weight steps (and the bias) of the tile
 // are read from their copy in shared memory (`dw_s`, `bias_s`: this tile's BN floats, indexed by the
 // column inside the tile) with broadcast loads: no global-memory latency sits in the conversion loop.
@@ -342,11 +343,11 @@ template <bool kDebugAcc>
 __device__ __forceinline__ uint32_t epilogue_tile_stream(const GemmParams &p, const CUtensorMap *tmY, uint32_t tmem_row,
                                                          long long m_row0, int n0, float dxr, uint32_t staging,
                                                          const float *dw_s, const float *bias_s, uint32_t nboxes,
-                                                         int lane, int col_half, int zr, bool two_boxes)
+                                                         int lane, int c_begin, int c_stride, int zr, bool two_boxes)
 {
     const long long m = m_row0 + lane;
     const bool row_ok = m < p.M;
-    for (int c0 = col_half * kEpiStepCols; c0 < p.BN; c0 += 2 * kEpiStepCols) {
+    for (int c0 = c_begin; c0 < p.BN; c0 += c_stride) {
         const int n_first = n0 + c0;
         uint32_t v0[32], v1[32];
         tmem_ld_32x32(tmem_row + c0, v0);
@@ -399,9 +400,114 @@ __device__ __forceinline__ uint32_t epilogue_tile_stream(const GemmParams &p, co
     return nboxes;
 }
 
+// --- epilogue in two teams -----------------------------------------------------------------------
+//
+// The arithmetic of a 64-column step (int32 -> binary32, two multiplies, conversion to binary16) keeps a
+// scheduler's issue port busy for about 400 cycles per warp, and around it sit waits that nothing else
+// of the same warp can fill (TMEM data arriving, the fence, the store issue, the previous store reading
+// its box).  With all eight warps on one tile, two warps per scheduler run those steps side by side and
+// the tile's epilogue lasts as long as the main loop of a K = 768 tile; the MMA thread then waits for
+// the accumulator.  In team mode the eight warps form two teams of four (one warp per TMEM lane quarter
+// and per scheduler); team b drains accumulator b, i.e. every second tile of the CTA, all 64-column
+// steps of it.  A tile's epilogue takes longer, but it has two main loops' time to finish, and one
+// team's waits are filled by the other team's arithmetic.  Used when a CTA has several tiles and the
+// main loop of a tile is short (K <= 384), i.e. where the epilogue sets the pace: 7-8 % on such layers
+// with many rows; layers with a long main loop are bounded elsewhere and gain nothing.
+//
+// The team's copy of the tile's weight steps (and bias) lives in scale buffer b; a named barrier over
+// the team's 128 threads publishes it (together with the vote on the bounded waits, so that the four
+// warps leave the loop together or not at all) and a second one, at the end of the tile, keeps the
+// next tile's values from overwriting it while a slower warp still reads.
+__device__ __forceinline__ bool team_all(bool pred, int team)
+{
+    uint32_t r;
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p, q;\n\t"
+        "setp.ne.u32 q, %1, 0;\n\t"
+        "bar.red.and.pred p, %2, 128, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t"
+        "}"
+        : "=r"(r)
+        : "r"(static_cast<uint32_t>(pred)), "r"(1 + team)
+        : "memory");
+    return r != 0u;
+}
+__device__ __forceinline__ void team_sync(int team) { asm volatile("bar.sync %0, 128;" ::"r"(1 + team) : "memory"); }
+
+// The CTA's tiles in the order the MMA thread produces them.
+struct StreamCursor {
+    int tile, total, step, n_tiles;
+    __device__ bool valid() const { return tile < total; }
+    __device__ void advance() { tile += step; }
+    __device__ int m_tile() const { return tile / n_tiles; }
+    __device__ int n_tile() const { return tile % n_tiles; }
+};
+template <bool kDebugAcc, class Cursor>
+__device__ __forceinline__ void epilogue_team_loop(const GemmParams &p, const CUtensorMap *tmY, Cursor cur, uint32_t tmem_base,
+                                                   uint32_t tfull_bar0, uint32_t tempty_bar0, float *scale_s,
+                                                   uint32_t staging, bool two_boxes, volatile uint32_t *abort_flag,
+                                                   int warp, int lane)
+{
+    const int quarter = warp & 3;                       // TMEM lanes [32*quarter, 32*quarter+32)
+    const int team = (warp - 2) >> 2;                   // = the accumulator buffer this team drains
+    const int tt = static_cast<int>(threadIdx.x) - 64 - team * 128;   // 0 .. 127 inside the team
+    float *dw_buf = scale_s + team * kMaxBN;
+    float *bias_buf = scale_s + (2 + team) * kMaxBN;
+    const uint32_t tfull = tfull_bar0 + 8u * team, tempty = tempty_bar0 + 8u * team;
+    if (team == 1 && cur.valid()) cur.advance();        // team 1 starts at the CTA's second tile
+    float dw_next[2] = {0.0f, 0.0f}, bias_next[2] = {0.0f, 0.0f};
+    auto fetch_scales = [&](const Cursor &c) {
+        if (!c.valid()) return;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int col = tt + 128 * h;
+            if (col < p.BN) {
+                const int n = c.n_tile() * p.BN + col;
+                dw_next[h] = __ldg(p.dw + n);
+                if (p.has_bias) bias_next[h] = __ldg(p.bias + n);
+            }
+        }
+    };
+    fetch_scales(cur);
+    uint32_t tphase = 0, nboxes = 0;
+    while (cur.valid()) {                               // the same for every thread of the team
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int col = tt + 128 * h;
+            if (col < p.BN) {
+                dw_buf[col] = dw_next[h];
+                if (p.has_bias) bias_buf[col] = bias_next[h];
+            }
+        }
+        const int m_tile = cur.m_tile(), n_tile = cur.n_tile();
+        cur.advance();
+        if (cur.valid()) cur.advance();                 // the team's next tile: its scales stay in flight during this one
+        fetch_scales(cur);
+        const long long m_row0 = static_cast<long long>(m_tile) * kBM + quarter * 32;
+        const long long m = m_row0 + lane;
+        const int t_row = (m < p.M) ? static_cast<int>(m % p.T) : 0;
+        const float dxr = (m < p.M) ? __ldg(p.dx + t_row) : 0.0f;
+        const int zr = (p.zp != nullptr) ? __ldg(p.zp + t_row) : 0;
+        bool got = mbar_wait(tfull, tphase, abort_flag, p.status);
+        got = team_all(got, team);                      // also: the team's scale copies are complete and visible
+        if (!got) break;
+        tc_fence_after_sync();
+        const uint32_t tmem_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(team) * kMaxBN;
+        nboxes = epilogue_tile_stream<kDebugAcc>(p, tmY, tmem_row, m_row0, n_tile * p.BN, dxr, staging, dw_buf,
+                                                 p.has_bias ? bias_buf : nullptr, nboxes, lane, 0, kEpiStepCols, zr, two_boxes);
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(tempty);
+        tphase ^= 1u;
+        team_sync(team);                                // every warp of the team is done reading the scale copies
+    }
+    if (lane == 0) bulk_wait_group<0>();                // all of this thread's stores have completed
+}
+
 // --- the kernel ---------------------------------------------------------------------------------
 
-template <bool kDebugAcc>
+template <bool kDebugAcc, bool kTeams = false>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 ptq_gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
                         const __grid_constant__ CUtensorMap tmY, const GemmParams p)
@@ -438,7 +544,7 @@ ptq_gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         }
         for (uint32_t b = 0; b < 2; ++b) {
             mbar_init(tfull_bar(b), 1);
-            mbar_init(tempty_bar(b), kNumEpiWarps);
+            mbar_init(tempty_bar(b), kTeams ? kNumEpiWarps / 2 : kNumEpiWarps);   // in team mode one team drains a buffer
         }
         mbar_init(scale_bar, kNumEpiWarps);
         *abort_flag = 0u;
@@ -531,6 +637,13 @@ ptq_gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                 if (buf == 0u) bphase ^= 1u;
             }
         }
+    } else if (kTeams) {
+        // ------------------------------------------------------------------ epilogue warps, two teams (TMA stores only)
+        const StreamCursor cur{static_cast<int>(blockIdx.x), total_tiles, static_cast<int>(gridDim.x), p.n_tiles};
+        epilogue_team_loop<kDebugAcc>(p, &tmY, cur, tmem_base, tfull_bar(0), tempty_bar(0),
+                                      reinterpret_cast<float *>(smem_raw + scale_off),
+                                      staging_base + static_cast<uint32_t>(warp - 2) * static_cast<uint32_t>(p.boxes) * kStreamStagingPerWarp,
+                                      two_boxes, abort_flag, warp, lane);
     } else {
         // ------------------------------------------------------------------ epilogue warps
         const int quarter = warp & 3;                // TMEM lanes [32*quarter, 32*quarter+32)
@@ -582,7 +695,7 @@ ptq_gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                 const float *dw_s = scale_s + (it & 1u) * kMaxBN;
                 const float *bias_s = p.has_bias ? scale_s + (2u + (it & 1u)) * kMaxBN : nullptr;
                 nboxes = epilogue_tile_stream<kDebugAcc>(p, &tmY, tmem_row, m_row0, n_tile * p.BN, dxr, staging, dw_s,
-                                                         bias_s, nboxes, lane, col_half, zr, two_boxes);
+                                                         bias_s, nboxes, lane, col_half * kEpiStepCols, 2 * kEpiStepCols, zr, two_boxes);
             } else {
                 nboxes = epilogue_tile<kDebugAcc, false, kStreamBox64>(p, &tmY, tmem_row, m_row0, n_tile * p.BN, dxr,
                                                                        staging, nboxes, lane, col_half, zr);
@@ -853,7 +966,7 @@ ptq_gemm_dequant_panel_kernel(const __grid_constant__ CUtensorMap tmA, const __g
             const float *dw_s = scale_s + (it & 1u) * kMaxBN;
             const float *bias_s = p.has_bias ? scale_s + (2u + (it & 1u)) * kMaxBN : nullptr;
             nboxes = epilogue_tile_stream<kDebugAcc>(p, &tmY, tmem_row, m_row0, n_tile * p.BN, dxr, staging, dw_s, bias_s,
-                                                     nboxes, lane, col_half, zr, two_boxes);
+                                                     nboxes, lane, col_half * kEpiStepCols, 2 * kEpiStepCols, zr, two_boxes);
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(tempty_bar(buf));
@@ -1072,8 +1185,8 @@ ptq_gemm_dequant_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __gr
             const uint32_t tmem_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * kMaxBN;
             if (p.use_tma_store)
                 nboxes = epilogue_tile_stream<kDebugAcc>(p, &tmY, tmem_row, m_row0, n_tile * p.BN, dxr, staging,
-                                                         scale_s + (it & 1u) * kMaxBN, nullptr, nboxes, lane, col_half, 0,
-                                                         false);
+                                                         scale_s + (it & 1u) * kMaxBN, nullptr, nboxes, lane,
+                                                         col_half * kEpiStepCols, 2 * kEpiStepCols, 0, false);
             else
                 nboxes = epilogue_tile<kDebugAcc, false, kStreamBox64>(p, &tmY, tmem_row, m_row0, n_tile * p.BN, dxr, staging,
                                                                        nboxes, lane, col_half);
