@@ -210,6 +210,18 @@ ptq_status_t ptq_linear_gemm_dequant(const ptq_linear_t *h, const void *q_int8, 
 int ptq_linear_code_pitch(const ptq_linear_t *h);
 
 /*
+ * Which G1 + E1 kernel (Sec. 5.1; Appendix B.1, parts 3-4) a forward pass over B images takes on the
+ * default path, assuming a 16-byte aligned y with N % 8 == 0 (otherwise always the first):
+ *   0  ptq_gemm_dequant_kernel          operand stages streamed per tile, eight epilogue warps per tile
+ *   1  ptq_gemm_dequant_kernel, teams   same, the epilogue warps in two teams, one per accumulator
+ *                                       (K <= 384 and at least four tiles per SM)
+ *   2  ptq_gemm_dequant_panel_kernel    the codes of a row panel resident in shared memory for a group
+ *                                       of N tiles (512 <= K <= 768, several N tiles, many tiles per SM)
+ * Returns -1 for a NULL handle or B < 1.  All variants produce the same bits.
+ */
+int ptq_linear_gemm_variant(const ptq_linear_t *h, int B);
+
+/*
  * Forward pass with parity taps.  Same as ptq_linear_forward, and additionally writes
  *   q_int8_out     device, [B,T,K] dense int8 codes of Q1, or NULL
  *                  (with PTQ_FLAG_FUSED_PROLOGUE the codes never exist in memory; they are then

@@ -62,6 +62,8 @@ def load_library() -> ctypes.CDLL:
     L.ptq_linear_workspace_bytes.argtypes = [vp, ci, cu]
     L.ptq_linear_forward.restype = ci
     L.ptq_linear_forward.argtypes = [vp, vp, ci, vp, vp, sz, cu, vp]
+    L.ptq_linear_gemm_variant.restype = ci
+    L.ptq_linear_gemm_variant.argtypes = [vp, ci]
     L.ptq_linear_forward_static.restype = ci
     L.ptq_linear_forward_static.argtypes = [vp, vp, ci, vp, vp]
     L.ptq_linear_workspace_bytes_dynamic.restype = sz
@@ -311,6 +313,10 @@ class PtqLinear:
 
     def code_pitch(self) -> int:
         return int(self._L.ptq_linear_code_pitch(self._h))
+
+    def gemm_variant(self, B: int) -> int:
+        """``ptq_linear_gemm_variant``: 0 streaming kernel, 1 streaming with two epilogue teams, 2 panel kernel."""
+        return int(self._L.ptq_linear_gemm_variant(self._h, int(B)))
 
     def gemm_dequant(self, q, B: int, y=None, stream=None):
         """``ptq_linear_gemm_dequant``: int8 codes [B*T, code_pitch()] -> y fp16 [B,T,N]."""

@@ -382,6 +382,13 @@ bool plan_panel(const ptq_linear *h, ptq::GemmParams &p, bool tma_store)
     return true;
 }
 
+// Whether the streaming kernel runs its epilogue in two teams: short main loop (K <= 384) and several tiles per CTA.
+bool gemm_teams(const ptq_linear *h, const ptq::GemmParams &p, bool tma_store, bool short_k)
+{
+    const long long tiles = static_cast<long long>(p.m_tiles) * p.n_tiles;
+    return PTQ_GEMM_TEAMS && tma_store && short_k && tiles >= static_cast<long long>(PTQ_GEMM_TEAM_MIN_ROUNDS) * h->num_sms;
+}
+
 // G1+E1 launch on codes [M, Kpad] at `codes`.
 // dx_rows != nullptr: the steps are per ROW (dynamic comparator), i.e. dx = dx_rows and T = M.
 ptq_status_t launch_gemm(const ptq_linear *h, const void *codes, long long M, void *y, void *acc_out,
@@ -463,8 +470,7 @@ ptq_status_t launch_gemm(const ptq_linear *h, const void *codes, long long M, vo
     const long long tiles = static_cast<long long>(p.m_tiles) * p.n_tiles;
     // Short main loop (K <= 384) and several tiles per CTA: the epilogue sets the pace and runs in two teams of
     // four warps, one per accumulator; otherwise all eight warps share every tile (shorter latency of a tile).
-    const bool teams = PTQ_GEMM_TEAMS && tma_store && short_k &&
-                       tiles >= static_cast<long long>(PTQ_GEMM_TEAM_MIN_ROUNDS) * h->num_sms;
+    const bool teams = gemm_teams(h, p, tma_store, short_k);
     const bool dbg = acc_out != nullptr;
     if (plan_panel(h, p, tma_store)) {
         // several N tiles and 512 <= K <= 768: the codes of a row panel stay in shared memory for `group` tiles
@@ -865,6 +871,23 @@ int ptq_linear_describe(const ptq_linear_t *h, char *buf, int buf_bytes)
 }
 
 int ptq_linear_code_pitch(const ptq_linear_t *h) { return h ? h->Kpad : 0; }
+
+int ptq_linear_gemm_variant(const ptq_linear_t *h, int B)
+{
+    if (!h || B < 1) return -1;
+    const long long M = static_cast<long long>(B) * h->T;
+    if (h->N % 8 != 0) return 0;
+    ptq::GemmParams p = {};
+    p.BN = h->BN;
+    p.n_tiles = h->n_tiles;
+    p.m_tiles = static_cast<int>((M + ptq::kBM - 1) / ptq::kBM);
+    p.k_blocks = h->k_blocks;
+    p.has_bias = h->has_bias ? 1 : 0;
+    const bool short_k = h->k_blocks <= PTQ_GEMM_SHORT_K_BLOCKS;
+    p.boxes = short_k ? 2 : 1;
+    if (plan_panel(h, p, true)) return 2;
+    return gemm_teams(h, p, true, short_k) ? 1 : 0;
+}
 
 ptq_status_t ptq_linear_gemm_dequant(const ptq_linear_t *h, const void *q_int8, int B, void *y_fp16, void *stream)
 {

@@ -73,6 +73,7 @@ def test_create_rejects_bad_arguments_before_touching_a_device(lib):
 def test_null_handles_are_refused_not_dereferenced(lib):
     assert lib.ptq_linear_workspace_bytes(None, 4, 0) == 0
     assert lib.ptq_linear_fused_supported(None) == 0
+    assert lib.ptq_linear_gemm_variant(None, 1) == -1
     assert lib.ptq_linear_forward(None, None, 1, None, None, 0, 0, None) == 1
     assert lib.ptq_quantize(None, None, 1, None, None) == 1
     assert lib.ptq_linear_device_status(None) == 1

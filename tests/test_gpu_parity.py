@@ -347,3 +347,17 @@ def test_forward_argument_errors_return_codes(env):
     layer.device_status()
     assert_y_close(y.cpu().numpy().reshape(-1, spec.N),
                    oracle.linear_forward(x.reshape(-1, spec.K), spec.T, wq, dw, s, dx, bias), "after errors")
+
+
+def test_gemm_kernel_selection_covers_all_three_variants(env):
+    """The three GEMM kernels are all reached by the configured workloads (so the parity tests above compare each
+    of them with the oracle): streaming for one-tile layers and long main loops, the two-team epilogue for short
+    main loops with many tiles, the resident-panel kernel for the Vim-B in_proj."""
+    ptq, torch = env
+    want = {(0, 0): 0, (3, 0): 2, (3, 1): 0, (4, 0): 1, (4, 2): 1, (2, 0): 1, (2, 1): 0}
+    for (cfg, idx), variant in want.items():
+        spec = CFG[cfg][idx]
+        x, wq, dw, bias, s, dx = layer_inputs(spec, B=1)
+        layer = ptq.PtqLinear(wq, dw, s, dx, bias)
+        assert layer.gemm_variant(spec.B) == variant, (spec.name, spec.M, spec.K, spec.N, layer.gemm_variant(spec.B))
+        assert layer.gemm_variant(0) == -1
