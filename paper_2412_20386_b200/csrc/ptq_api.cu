@@ -377,6 +377,7 @@ bool plan_panel(const ptq_linear *h, ptq::GemmParams &p, bool tma_store)
     if (best_g < 2) return false;
     p.group = best_g;
     p.groups = (p.n_tiles + best_g - 1) / best_g;
+    p.fd_groups = ptq::make_fastdiv(static_cast<unsigned>(p.groups));
     p.b_stages = stages;
     p.b_stage_bytes = stage_bytes;
     return true;
@@ -443,6 +444,9 @@ ptq_status_t launch_gemm(const ptq_linear *h, const void *codes, long long M, vo
     p.y_vec8 = 0;   // this kernel always has a staging buffer; 16-byte alignment means TMA stores
     p.zp = h->d_zp;
     p.wsum = h->d_wsum;
+    p.fd_T = ptq::make_fastdiv(static_cast<unsigned>(p.T));
+    p.fd_n_tiles = ptq::make_fastdiv(static_cast<unsigned>(p.n_tiles));
+    p.fd_groups = ptq::make_fastdiv(1u);
 
     if (use_pair) {
         // enough 256-row tiles to occupy every CTA pair: cta_group::2 kernel (half the weight bytes per CTA)

@@ -67,6 +67,26 @@ constexpr int kGemmSmemBytes = gemm_smem_bytes(kStages, 1, 0);
 static_assert(kGemmSmemBytes <= 232448 && gemm_smem_bytes(kStages - 1, 2, 1) <= kGemmSmemBytes,
               "streaming GEMM kernel exceeds the shared memory of one CTA");
 
+// Division of a 32-bit number by a launch constant without a division: with magic = ceil(2^64 / d), the
+// high 64 bits of magic * n are floor(n / d) for every 32-bit n.  A runtime integer division is a chain of
+// some twenty dependent instructions; at the top of an epilogue loop, where the warp has nothing else to
+// issue, several of them cost hundreds of cycles per tile.
+struct FastDiv {
+    unsigned d;
+    unsigned long long magic;
+};
+__host__ __device__ inline FastDiv make_fastdiv(unsigned d)
+{
+    FastDiv f;
+    f.d = d;
+    f.magic = d > 1u ? 0xFFFFFFFFFFFFFFFFull / d + 1ull : 0ull;
+    return f;
+}
+__device__ __forceinline__ unsigned fd_div(unsigned n, const FastDiv &f)
+{
+    return f.d == 1u ? n : static_cast<unsigned>(__umul64hi(f.magic, static_cast<unsigned long long>(n)));
+}
+
 struct GemmParams {
     long long M;
     int N, K, T;
@@ -95,6 +115,7 @@ struct GemmParams {
     // units cover a panel; the weight ring has `b_stages` slots of `b_stage_bytes` (= BN * 128) each.
     int group, groups;
     int b_stages, b_stage_bytes;
+    FastDiv fd_T, fd_n_tiles, fd_groups;   // divisors T, n_tiles, groups (the GEMM kernels' loops)
 };
 
 // --- epilogue helpers -------------------------------------------------------------------------
@@ -400,6 +421,28 @@ __device__ __forceinline__ uint32_t epilogue_tile_stream(const GemmParams &p, co
     return nboxes;
 }
 
+// The activation step (and, on asymmetric layers, the zero offset) of this thread's row of row tile `m_tile`.
+// The epilogue loops request it one tile ahead, so that neither the load's latency nor the modulo sits between
+// two tiles.  B*T < 2^31 (checked at the boundary), so the row index fits 32 bits.
+struct RowStep {
+    float dx;
+    int z;
+};
+__device__ __forceinline__ RowStep load_row_step(const GemmParams &p, int m_tile, int quarter, int lane)
+{
+    // Unconditional loads from clamped indices: a load under a condition is followed by a select that waits for
+    // it, which would put the load's latency back into the loop.  Rows beyond M are never stored, so what they
+    // get does not matter.
+    RowStep r = {0.0f, 0};
+    long long m = static_cast<long long>(m_tile) * kBM + quarter * 32 + lane;
+    if (m >= p.M) m = p.M - 1;
+    const unsigned mu = static_cast<unsigned>(m);
+    const unsigned t = mu - fd_div(mu, p.fd_T) * p.fd_T.d;
+    r.dx = __ldg(p.dx + t);
+    if (p.zp != nullptr) r.z = __ldg(p.zp + t);
+    return r;
+}
+
 // --- epilogue in two teams -----------------------------------------------------------------------
 //
 // The arithmetic of a 64-column step (int32 -> binary32, two multiplies, conversion to binary16) keeps a
@@ -438,11 +481,13 @@ __device__ __forceinline__ void team_sync(int team) { asm volatile("bar.sync %0,
 // The CTA's tiles in the order the MMA thread produces them.
 struct StreamCursor {
     int tile, total, step, n_tiles;
+    FastDiv fd;
     __device__ bool valid() const { return tile < total; }
     __device__ void advance() { tile += step; }
-    __device__ int m_tile() const { return tile / n_tiles; }
-    __device__ int n_tile() const { return tile % n_tiles; }
+    __device__ int m_tile() const { return static_cast<int>(fd_div(static_cast<unsigned>(tile), fd)); }
+    __device__ int n_tile() const { return tile - m_tile() * n_tiles; }
 };
+
 template <bool kDebugAcc, class Cursor>
 __device__ __forceinline__ void epilogue_team_loop(const GemmParams &p, const CUtensorMap *tmY, Cursor cur, uint32_t tmem_base,
                                                    uint32_t tfull_bar0, uint32_t tempty_bar0, float *scale_s,
@@ -458,18 +503,18 @@ __device__ __forceinline__ void epilogue_team_loop(const GemmParams &p, const CU
     if (team == 1 && cur.valid()) cur.advance();        // team 1 starts at the CTA's second tile
     float dw_next[2] = {0.0f, 0.0f}, bias_next[2] = {0.0f, 0.0f};
     auto fetch_scales = [&](const Cursor &c) {
-        if (!c.valid()) return;
+        // unconditional loads from clamped indices (see load_row_step); past the last tile the values are not used
+        const int n0 = c.valid() ? c.n_tile() * p.BN : 0;
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
-            const int col = tt + 128 * h;
-            if (col < p.BN) {
-                const int n = c.n_tile() * p.BN + col;
-                dw_next[h] = __ldg(p.dw + n);
-                if (p.has_bias) bias_next[h] = __ldg(p.bias + n);
-            }
+            const int col = min(tt + 128 * h, p.BN - 1);
+            dw_next[h] = __ldg(p.dw + n0 + col);
+            if (p.has_bias) bias_next[h] = __ldg(p.bias + n0 + col);
         }
     };
     fetch_scales(cur);
+    RowStep rs_next = {0.0f, 0};
+    if (cur.valid()) rs_next = load_row_step(p, cur.m_tile(), quarter, lane);
     uint32_t tphase = 0, nboxes = 0;
     while (cur.valid()) {                               // the same for every thread of the team
 #pragma unroll
@@ -485,10 +530,9 @@ __device__ __forceinline__ void epilogue_team_loop(const GemmParams &p, const CU
         if (cur.valid()) cur.advance();                 // the team's next tile: its scales stay in flight during this one
         fetch_scales(cur);
         const long long m_row0 = static_cast<long long>(m_tile) * kBM + quarter * 32;
-        const long long m = m_row0 + lane;
-        const int t_row = (m < p.M) ? static_cast<int>(m % p.T) : 0;
-        const float dxr = (m < p.M) ? __ldg(p.dx + t_row) : 0.0f;
-        const int zr = (p.zp != nullptr) ? __ldg(p.zp + t_row) : 0;
+        const float dxr = rs_next.dx;
+        const int zr = rs_next.z;
+        if (cur.valid()) rs_next = load_row_step(p, cur.m_tile(), quarter, lane);
         bool got = mbar_wait(tfull, tphase, abort_flag, p.status);
         got = team_all(got, team);                      // also: the team's scale copies are complete and visible
         if (!got) break;
@@ -575,7 +619,7 @@ ptq_gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             uint32_t stage = 0, phase = 0, issued = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-                const int m_tile = tile / p.n_tiles;
+                const int m_tile = static_cast<int>(fd_div(static_cast<unsigned>(tile), p.fd_n_tiles));
                 const int n_tile = tile - m_tile * p.n_tiles;
                 for (int kb = 0; kb < p.k_blocks; ++kb) {
                     if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status)) {
@@ -639,7 +683,7 @@ ptq_gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         }
     } else if (kTeams) {
         // ------------------------------------------------------------------ epilogue warps, two teams (TMA stores only)
-        const StreamCursor cur{static_cast<int>(blockIdx.x), total_tiles, static_cast<int>(gridDim.x), p.n_tiles};
+        const StreamCursor cur{static_cast<int>(blockIdx.x), total_tiles, static_cast<int>(gridDim.x), p.n_tiles, p.fd_n_tiles};
         epilogue_team_loop<kDebugAcc>(p, &tmY, cur, tmem_base, tfull_bar(0), tempty_bar(0),
                                       reinterpret_cast<float *>(smem_raw + scale_off),
                                       staging_base + static_cast<uint32_t>(warp - 2) * static_cast<uint32_t>(p.boxes) * kStreamStagingPerWarp,
@@ -654,11 +698,11 @@ ptq_gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         // The weight step (and bias) of one column of tile `tile`: fetched into registers one tile ahead ...
         float dw_next = 0.0f, bias_next = 0.0f;
         auto fetch_scales = [&](int tile) {
-            if (tile < total_tiles && et < p.BN) {
-                const int n = (tile % p.n_tiles) * p.BN + et;
-                dw_next = __ldg(p.dw + n);
-                if (p.has_bias) bias_next = __ldg(p.bias + n);
-            }
+            // unconditional loads from clamped indices (see load_row_step); past the last tile the values are not used
+            const unsigned tl = tile < total_tiles ? static_cast<unsigned>(tile) : 0u;
+            const int n = static_cast<int>(tl - fd_div(tl, p.fd_n_tiles) * p.fd_n_tiles.d) * p.BN + min(et, p.BN - 1);
+            dw_next = __ldg(p.dw + n);
+            if (p.has_bias) bias_next = __ldg(p.bias + n);
         };
         // ... and published in buffer `b` once every warp is done with the tile that used that buffer last
         auto publish_scales = [&](uint32_t b) {
@@ -674,15 +718,17 @@ ptq_gemm_dequant_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             fetch_scales(blockIdx.x);
             publish_scales(0u);
         }
+        RowStep rs_next = load_row_step(p, static_cast<int>(fd_div(blockIdx.x, p.fd_n_tiles)), quarter, lane);
         for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++it) {
-            if (p.use_tma_store) fetch_scales(tile + static_cast<int>(gridDim.x));   // in flight during this tile
-            const int m_tile = tile / p.n_tiles;
+            const int tile_next = tile + static_cast<int>(gridDim.x);
+            if (p.use_tma_store) fetch_scales(tile_next);                            // in flight during this tile
+            const int m_tile = static_cast<int>(fd_div(static_cast<unsigned>(tile), p.fd_n_tiles));
             const int n_tile = tile - m_tile * p.n_tiles;
             const long long m_row0 = static_cast<long long>(m_tile) * kBM + quarter * 32;
-            const long long m = m_row0 + lane;
-            const int t_row = (m < p.M) ? static_cast<int>(m % p.T) : 0;
-            const float dxr = (m < p.M) ? __ldg(p.dx + t_row) : 0.0f;
-            const int zr = (p.zp != nullptr) ? __ldg(p.zp + t_row) : 0;
+            const float dxr = rs_next.dx;
+            const int zr = rs_next.z;
+            if (tile_next < total_tiles)
+                rs_next = load_row_step(p, static_cast<int>(fd_div(static_cast<unsigned>(tile_next), p.fd_n_tiles)), quarter, lane);
             bool got = true;
             // every epilogue warp has written its share of this tile's scale copies (arrival `it` of the barrier)
             if (p.use_tma_store) got = mbar_wait(scale_bar, it & 1u, abort_flag, p.status);
@@ -812,7 +858,8 @@ ptq_gemm_dequant_panel_kernel(const __grid_constant__ CUtensorMap tmA, const __g
 
     const int units = p.m_tiles * p.groups;
     // unit u -> panel u / groups, N tiles [first, first + count)
-    auto unit_first = [&](int u) { return (u % p.groups) * p.group; };
+    auto unit_panel = [&](int u) { return static_cast<int>(fd_div(static_cast<unsigned>(u), p.fd_groups)); };
+    auto unit_first = [&](int u) { return (u - unit_panel(u) * p.groups) * p.group; };
     auto unit_count = [&](int u) {
         const int left = p.n_tiles - unit_first(u);
         return left < p.group ? left : p.group;
@@ -825,7 +872,7 @@ ptq_gemm_dequant_panel_kernel(const __grid_constant__ CUtensorMap tmA, const __g
             int a_kb_issued = 0;                 // panel k-blocks issued for the unit in progress
             bool ok = true;
             for (int unit = blockIdx.x; unit < units && ok; unit += gridDim.x, uph ^= 1u) {
-                const int m_tile = unit / p.groups;
+                const int m_tile = unit_panel(unit);
                 const int n_first = unit_first(unit), n_count = unit_count(unit);
                 a_kb_issued = 0;
                 for (int j = 0; j < n_count && ok; ++j) {
@@ -924,11 +971,9 @@ ptq_gemm_dequant_panel_kernel(const __grid_constant__ CUtensorMap tmA, const __g
         float *scale_s = reinterpret_cast<float *>(smem_raw + scale_off);   // [2][BN] steps, then [2][BN] bias
         float dw_next = 0.0f, bias_next = 0.0f;
         auto fetch_scales = [&](int n_tile) {
-            if (et < p.BN) {
-                const int n = n_tile * p.BN + et;
-                dw_next = __ldg(p.dw + n);
-                if (p.has_bias) bias_next = __ldg(p.bias + n);
-            }
+            const int n = n_tile * p.BN + min(et, p.BN - 1);      // unconditional, clamped (see load_row_step)
+            dw_next = __ldg(p.dw + n);
+            if (p.has_bias) bias_next = __ldg(p.bias + n);
         };
         auto publish_scales = [&](uint32_t b) {
             if (et < p.BN) {
@@ -940,8 +985,9 @@ ptq_gemm_dequant_panel_kernel(const __grid_constant__ CUtensorMap tmA, const __g
         };
         uint32_t buf = 0, bphase = 0, nboxes = 0, it = 0;
         int unit = blockIdx.x, j = 0;
-        if (unit < units) fetch_scales(unit_first(unit));
+        fetch_scales(unit < units ? unit_first(unit) : 0);
         publish_scales(0u);
+        RowStep rs_next = load_row_step(p, unit < units ? unit_panel(unit) : 0, quarter, lane);
         while (unit < units) {
             // the tile after this one: its scales are fetched now and stay in flight during this tile
             int next_unit = unit, next_j = j + 1;
@@ -949,14 +995,13 @@ ptq_gemm_dequant_panel_kernel(const __grid_constant__ CUtensorMap tmA, const __g
                 next_unit = unit + static_cast<int>(gridDim.x);
                 next_j = 0;
             }
-            if (next_unit < units) fetch_scales(unit_first(next_unit) + next_j);
-            const int m_tile = unit / p.groups;
+            fetch_scales(next_unit < units ? unit_first(next_unit) + next_j : 0);
+            const int m_tile = unit_panel(unit);
             const int n_tile = unit_first(unit) + j;
             const long long m_row0 = static_cast<long long>(m_tile) * kBM + quarter * 32;
-            const long long m = m_row0 + lane;
-            const int t_row = (m < p.M) ? static_cast<int>(m % p.T) : 0;
-            const float dxr = (m < p.M) ? __ldg(p.dx + t_row) : 0.0f;
-            const int zr = (p.zp != nullptr) ? __ldg(p.zp + t_row) : 0;
+            const float dxr = rs_next.dx;
+            const int zr = rs_next.z;
+            if (next_unit != unit && next_unit < units) rs_next = load_row_step(p, unit_panel(next_unit), quarter, lane);
             bool got = mbar_wait(scale_bar, it & 1u, abort_flag, p.status);
             got = got && mbar_wait(tfull_bar(buf), bphase, abort_flag, p.status);
             got = __all_sync(0xffffffffu, got);
