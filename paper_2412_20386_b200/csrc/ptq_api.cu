@@ -106,6 +106,22 @@ bool ranges_overlap(const void *a, size_t na, const void *b, size_t nb)
 
 }  // namespace
 
+// Tensor maps of the caller's buffers, remembered per handle: encoding one costs the host about as much as a
+// kernel launch, and a layer is normally called again and again with the same few buffers and batch sizes.
+// Keyed by everything the encoding depends on besides the layer (pointer, rows, box width); four entries
+// per kind, replaced in turn.  The lock is per handle and held for a lookup or an insertion only.
+struct MapCache {
+    struct Entry {
+        const void *ptr = nullptr;
+        long long rows = -1;
+        unsigned box_cols = 0;
+        CUtensorMap map;
+    };
+    Entry e[4];
+    unsigned next = 0;
+    std::mutex mu;
+};
+
 struct ptq_linear {
     int K = 0, N = 0, T = 0;
     int Kpad = 0;              // pitch of the codes workspace and of the padded weight: K rounded up to 16
@@ -132,6 +148,7 @@ struct ptq_linear {
     bool as_ok = false;
     int as_BN = 0, as_n_tiles = 0, as_w_stages = 0, as_w_stage_bytes = 0, as_staging = 0, as_smem = 0;
     CUtensorMap tmWas;
+    mutable MapCache codes_maps, y_maps;   // tensor maps of caller buffers seen so far
 };
 
 namespace {
@@ -150,6 +167,28 @@ ptq_status_t check_device(const ptq_linear *h)
     PTQ_CUDA(cudaGetDevice(&dev));
     if (dev != h->device)
         return fail(PTQ_ERR_CUDA, "handle belongs to device %d but device %d is current", h->device, dev);
+    return PTQ_OK;
+}
+
+// make_map_2d through a handle's cache.
+ptq_status_t cached_map_2d(MapCache &cache, CUtensorMap *map, CUtensorMapDataType dt, int elem_bytes, const void *ptr,
+                           unsigned long long cols, unsigned long long rows, unsigned long long pitch_bytes,
+                           unsigned box_cols, unsigned box_rows)
+{
+    std::lock_guard<std::mutex> lock(cache.mu);
+    for (const MapCache::Entry &e : cache.e)
+        if (e.ptr == ptr && e.rows == static_cast<long long>(rows) && e.box_cols == box_cols) {
+            *map = e.map;
+            return PTQ_OK;
+        }
+    const ptq_status_t st = make_map_2d(map, dt, elem_bytes, ptr, cols, rows, pitch_bytes, box_cols, box_rows);
+    if (st != PTQ_OK) return st;
+    MapCache::Entry &slot = cache.e[cache.next];
+    cache.next = (cache.next + 1u) % 4u;
+    slot.ptr = ptr;
+    slot.rows = static_cast<long long>(rows);
+    slot.box_cols = box_cols;
+    slot.map = *map;
     return PTQ_OK;
 }
 
@@ -396,9 +435,9 @@ ptq_status_t launch_gemm(const ptq_linear *h, const void *codes, long long M, vo
                          cudaStream_t stream, bool want_pair = false, const float *dx_rows = nullptr)
 {
     CUtensorMap tmA, tmY;
-    ptq_status_t st = make_map_2d(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, codes, static_cast<unsigned long long>(h->K),
-                                  static_cast<unsigned long long>(M), static_cast<unsigned long long>(h->Kpad),
-                                  ptq::kBK, ptq::kBM);
+    ptq_status_t st = cached_map_2d(h->codes_maps, &tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, codes,
+                                    static_cast<unsigned long long>(h->K), static_cast<unsigned long long>(M),
+                                    static_cast<unsigned long long>(h->Kpad), ptq::kBK, ptq::kBM);
     if (st != PTQ_OK) return st;
     const bool tma_store = (h->N % 8 == 0) && (reinterpret_cast<uintptr_t>(y) % 16 == 0);
     const int m_tiles_ = static_cast<int>((M + ptq::kBM - 1) / ptq::kBM);
@@ -408,9 +447,9 @@ ptq_status_t launch_gemm(const ptq_linear *h, const void *codes, long long M, vo
     const bool use_pair = want_pair && h->max_pairs > 0 && !h->has_bias &&
                           static_cast<long long>((m_tiles_ + 1) / 2) * h->n_tiles >= h->max_pairs;
     if (tma_store) {
-        st = make_map_2d(&tmY, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, y, static_cast<unsigned long long>(h->N),
-                         static_cast<unsigned long long>(M), static_cast<unsigned long long>(h->N) * 2,
-                         ptq::kStreamBoxCols, 32);
+        st = cached_map_2d(h->y_maps, &tmY, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, y, static_cast<unsigned long long>(h->N),
+                           static_cast<unsigned long long>(M), static_cast<unsigned long long>(h->N) * 2,
+                           ptq::kStreamBoxCols, 32);
         if (st != PTQ_OK) return st;
     } else {
         tmY = h->tmW;   // never dereferenced by the kernel in this mode
@@ -561,9 +600,9 @@ ptq_status_t launch_fused(const ptq_linear *h, const void *x, long long M, void 
     const bool aligned = (h->N % 8 == 0) && (reinterpret_cast<uintptr_t>(y) % 16 == 0);
     const bool tma_store = aligned && h->as_staging;
     if (tma_store) {
-        st = make_map_2d(&tmY, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, y, static_cast<unsigned long long>(h->N),
-                         static_cast<unsigned long long>(M), static_cast<unsigned long long>(h->N) * 2,
-                         ptq::kStoreBoxCols, 32);
+        st = cached_map_2d(h->y_maps, &tmY, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, y, static_cast<unsigned long long>(h->N),
+                           static_cast<unsigned long long>(M), static_cast<unsigned long long>(h->N) * 2,
+                           ptq::kStoreBoxCols, 32);
         if (st != PTQ_OK) return st;
     } else {
         tmY = h->tmWas;   // never dereferenced by the kernel in this mode
