@@ -214,7 +214,7 @@ int ptq_linear_code_pitch(const ptq_linear_t *h);
  * default path, assuming a 16-byte aligned y with N % 8 == 0 (otherwise always the first):
  *   0  ptq_gemm_dequant_kernel          operand stages streamed per tile, eight epilogue warps per tile
  *   1  ptq_gemm_dequant_kernel, teams   same, the epilogue warps in two teams, one per accumulator
- *                                       (K <= 384 and at least four tiles per SM)
+ *                                       (K <= 384 and at least three tiles per SM)
  *   2  ptq_gemm_dequant_panel_kernel    the codes of a row panel resident in shared memory for a group
  *                                       of N tiles (512 <= K <= 768, several N tiles, many tiles per SM)
  * Returns -1 for a NULL handle or B < 1.  All variants produce the same bits.

@@ -384,7 +384,7 @@ ptq_status_t launch_quantize_dynamic(const ptq_linear *h, const void *x, long lo
 #define PTQ_GEMM_TEAMS 1
 #endif
 #ifndef PTQ_GEMM_TEAM_MIN_ROUNDS
-#define PTQ_GEMM_TEAM_MIN_ROUNDS 4
+#define PTQ_GEMM_TEAM_MIN_ROUNDS 3
 #endif
 
 // Whether this launch takes the panel kernel (the codes of a row panel resident in shared memory for a
