@@ -570,6 +570,16 @@ def run_ours(args, specs, rank, world, local_rank):
                  "traffic": TRAFFIC.get((dom["kernel"], args.workload, dom["layer"].split(".")[-1]))
                  if args.scheme == "pts" else None})
 
+    # ---- what this GPU does for the bare data movements of the GEMM kernel (library probes, nothing else running)
+    scratch = torch.empty(448 << 20, dtype=torch.uint8, device=dev)
+    rates = {"store16_gbs": ptq.binding.probe(ptq.binding.PROBE_STORE16, scratch, 10),
+             "tma_store_epilogue_pattern_gbs": ptq.binding.probe(ptq.binding.PROBE_TMA_STORE, scratch, 10),
+             "operand_pull_l2_to_sm_gbs": ptq.binding.probe(ptq.binding.PROBE_OPERAND_PULL, scratch[:64 << 20], 10),
+             "empty_launch_us": ptq.binding.probe(ptq.binding.PROBE_LAUNCH, None, 500),
+             "empty_launch_pdl_us": ptq.binding.probe(ptq.binding.PROBE_LAUNCH_PDL, None, 500)}
+    rates = {k: round(v, 2) for k, v in rates.items()}
+    del scratch
+
     # ---- CPU oracle baseline on a bounded sample -------------------------------------------
     import oracle
     cpu_val, cpu_sample, cpu_secs, cpu_phases = time_oracle(specs, args.cpu_seconds)
@@ -604,6 +614,7 @@ def run_ours(args, specs, rank, world, local_rank):
                 "ms_per_step": ms_e2e},
         "gpu_launches": int(launches),
         "roofline": roof,
+        "measured_rates": rates,
         "kernels": [{k2: (round(v, 5) if isinstance(v, float) else v) for k2, v in k.items()} for k in kernels[:16]],
         "cpu_baseline": cpu,
     }

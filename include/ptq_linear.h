@@ -222,6 +222,24 @@ int ptq_linear_code_pitch(const ptq_linear_t *h);
 int ptq_linear_gemm_variant(const ptq_linear_t *h, int B);
 
 /*
+ * Measurement aid; the paper has no counterpart.  Times one of five stand-alone kernels that move bytes the way
+ * the GEMM + dequantization kernel does (Sec. 5.1; Appendix B.1, parts 3-4) but compute nothing, so that a
+ * roofline discussion can quote what THIS GPU does with nothing else running:
+ *   kind 0  16-byte stores over buf                                      result: GB/s written
+ *   kind 1  2-D TMA stores of 32 x 64 fp16 boxes over buf seen as y [M, 3072], in the epilogue's
+ *           tile order, one CTA per SM, eight warps                      result: GB/s written
+ *   kind 2  the operand stages of a [M, 768] x [3072, 768] problem (128 x 128 B + 256 x 128 B per k-block,
+ *           four stages per CTA) pulled by 2-D tiled TMA loads           result: GB/s delivered to the SMs
+ *   kind 3  an empty kernel, launches back to back                       result: microseconds per launch
+ *   kind 4  the same with programmatic dependent launch                  result: microseconds per launch
+ *   buf     device, 256-byte aligned scratch of `bytes` bytes (kinds 0-2; its contents are overwritten or
+ *           ignored; the last 256 bytes hold a status word); kinds 1 and 2 use as many 128-row tiles as fit
+ *   iters   timed launches (after three untimed ones), 1 .. 100000
+ * Allocates no device memory.  Synchronises the stream.  PTQ_ERR_SHAPE if buf is too small.
+ */
+ptq_status_t ptq_probe(int kind, void *buf, size_t bytes, int iters, double *result, void *stream);
+
+/*
  * Forward pass with parity taps.  Same as ptq_linear_forward, and additionally writes
  *   q_int8_out     device, [B,T,K] dense int8 codes of Q1, or NULL
  *                  (with PTQ_FLAG_FUSED_PROLOGUE the codes never exist in memory; they are then

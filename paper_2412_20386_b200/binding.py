@@ -62,6 +62,8 @@ def load_library() -> ctypes.CDLL:
     L.ptq_linear_workspace_bytes.argtypes = [vp, ci, cu]
     L.ptq_linear_forward.restype = ci
     L.ptq_linear_forward.argtypes = [vp, vp, ci, vp, vp, sz, cu, vp]
+    L.ptq_probe.restype = ci
+    L.ptq_probe.argtypes = [ci, vp, sz, ci, ctypes.POINTER(ctypes.c_double), vp]
     L.ptq_linear_gemm_variant.restype = ci
     L.ptq_linear_gemm_variant.argtypes = [vp, ci]
     L.ptq_linear_forward_static.restype = ci
@@ -148,6 +150,18 @@ def _scratch(nbytes: int, device, stream):
 
 def kernel_launch_count() -> int:
     return int(load_library().ptq_kernel_launch_count())
+
+
+PROBE_STORE16, PROBE_TMA_STORE, PROBE_OPERAND_PULL, PROBE_LAUNCH, PROBE_LAUNCH_PDL = 0, 1, 2, 3, 4
+
+
+def probe(kind: int, buf=None, iters: int = 20, stream=None) -> float:
+    """``ptq_probe``: GB/s (kinds 0-2, over the device uint8 tensor ``buf``) or microseconds per launch (kinds 3-4)."""
+    L = load_library()
+    out = ctypes.c_double(0.0)
+    ptr, nbytes = (None, 0) if buf is None else (buf.data_ptr(), buf.numel() * buf.element_size())
+    _check(L.ptq_probe(int(kind), ptr, nbytes, int(iters), ctypes.byref(out), _stream_ptr(stream)))
+    return float(out.value)
 
 
 class PtqLinear:

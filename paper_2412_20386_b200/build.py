@@ -18,7 +18,7 @@ _CSRC = os.path.join(_HERE, "csrc")
 _SO = os.path.join(_HERE, "libptq_linear.so")
 _SOURCES = ["ptq_api.cu"]
 _DEPS = ["ptq_api.cu", "ptq_gemm.cuh", "ptq_fused.cuh", "ptq_quantize.cuh", "ptq_quantize_dynamic.cuh",
-         "ptq_calibrate.cuh", "ptx_sm100.cuh",
+         "ptq_calibrate.cuh", "ptq_probe.cuh", "ptx_sm100.cuh",
          os.path.join("..", "..", "include", "ptq_linear.h")]
 
 

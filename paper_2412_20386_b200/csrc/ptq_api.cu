@@ -19,6 +19,7 @@
 #include "ptq_calibrate.cuh"
 #include "ptq_fused.cuh"
 #include "ptq_gemm.cuh"
+#include "ptq_probe.cuh"
 #include "ptq_quantize.cuh"
 #include "ptq_quantize_dynamic.cuh"
 
@@ -1153,6 +1154,99 @@ ptq_status_t ptq_linear_selftest_wait_timeout(const ptq_linear_t *h, unsigned li
     st = body();
     cudaFree(d_out);
     return st;
+}
+
+ptq_status_t ptq_probe(int kind, void *buf, size_t bytes, int iters, double *result, void *stream)
+{
+    if (!result) return fail(PTQ_ERR_NULL, "probe: result must not be NULL");
+    *result = 0.0;
+    if (kind < ptq::kProbeStore16 || kind > ptq::kProbeLaunchPdl) return fail(PTQ_ERR_VALUE, "probe: unknown kind %d", kind);
+    if (iters < 1 || iters > 100000) return fail(PTQ_ERR_VALUE, "probe: iters must be in [1, 100000] (got %d)", iters);
+    const bool moves_bytes = kind <= ptq::kProbeOperandPull;
+    if (moves_bytes && !buf) return fail(PTQ_ERR_NULL, "probe: buf must not be NULL for this kind");
+    if (moves_bytes && reinterpret_cast<uintptr_t>(buf) % 256) return fail(PTQ_ERR_ALIGN, "probe: buf must be 256-byte aligned");
+    int dev = -1, sms = 0, major = 0, minor = 0;
+    PTQ_CUDA(cudaGetDevice(&dev));
+    PTQ_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    PTQ_CUDA(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
+    PTQ_CUDA(cudaDeviceGetAttribute(&minor, cudaDevAttrComputeCapabilityMinor, dev));
+    if (major != 10 || minor != 0)
+        return fail(PTQ_ERR_ARCH, "device %d is compute capability %d.%d; this library needs 10.0 (sm_100a)", dev, major, minor);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    constexpr size_t kTail = 256;                      // the last 256 bytes of buf hold the kernels' status word
+    constexpr int N = 3072, K = 768;                   // the Vim-B in_proj shape: y [M, 3072] fp16, codes [M, 768], weights [3072, 768]
+    unsigned char *base = static_cast<unsigned char *>(buf);
+    unsigned *status = moves_bytes ? reinterpret_cast<unsigned *>(base + (bytes >= kTail ? bytes - kTail : 0)) : nullptr;
+    double moved = 0.0;                                // bytes per launch
+    int grid = sms, m_tiles = 0;
+    CUtensorMap tm0, tm1;
+    if (kind == ptq::kProbeStore16) {
+        if (bytes < kTail + (1u << 20)) return fail(PTQ_ERR_SHAPE, "probe: buf too small (%zu bytes)", bytes);
+        moved = static_cast<double>((bytes - kTail) / 16 * 16);
+        grid = sms * 32;
+    } else if (kind == ptq::kProbeTmaStore) {
+        m_tiles = static_cast<int>((bytes - (bytes >= kTail ? kTail : bytes)) / (static_cast<size_t>(N) * 2 * ptq::kBM));
+        if (m_tiles < 1) return fail(PTQ_ERR_SHAPE, "probe: buf too small (%zu bytes)", bytes);
+        if (m_tiles > 4096) m_tiles = 4096;
+        ptq_status_t st = make_map_2d(&tm0, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, base, N, static_cast<unsigned long long>(m_tiles) * ptq::kBM,
+                                      static_cast<unsigned long long>(N) * 2, 64, 32);
+        if (st != PTQ_OK) return st;
+        moved = static_cast<double>(m_tiles) * ptq::kBM * N * 2;
+        PTQ_CUDA(cudaFuncSetAttribute(ptq::ptq_probe_tma_store_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 8 * ptq::kProbeBoxBytes));
+    } else if (kind == ptq::kProbeOperandPull) {
+        const size_t w_bytes = static_cast<size_t>(N) * K;
+        if (bytes < kTail + w_bytes + static_cast<size_t>(ptq::kBM) * K) return fail(PTQ_ERR_SHAPE, "probe: buf too small (%zu bytes)", bytes);
+        m_tiles = static_cast<int>((bytes - kTail - w_bytes) / (static_cast<size_t>(ptq::kBM) * K));
+        if (m_tiles > 4096) m_tiles = 4096;
+        ptq_status_t st = make_map_2d(&tm0, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, base + w_bytes, K, static_cast<unsigned long long>(m_tiles) * ptq::kBM, K, 128, 128);
+        if (st == PTQ_OK) st = make_map_2d(&tm1, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, base, K, N, K, 128, 256);
+        if (st != PTQ_OK) return st;
+        moved = static_cast<double>(m_tiles) * (N / 256) * (K / 128) * ptq::kProbeStageBytes;
+        PTQ_CUDA(cudaFuncSetAttribute(ptq::ptq_probe_operand_pull_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      4 * ptq::kProbeStageBytes + 128));
+    }
+    if (status) PTQ_CUDA(cudaMemsetAsync(status, 0, sizeof(unsigned), s));
+    auto launch = [&]() -> cudaError_t {
+        switch (kind) {
+            case ptq::kProbeStore16:
+                ptq::ptq_probe_store16_kernel<<<grid, 256, 0, s>>>(reinterpret_cast<uint4 *>(base), static_cast<unsigned long long>(moved / 16));
+                break;
+            case ptq::kProbeTmaStore:
+                ptq::ptq_probe_tma_store_kernel<<<sms, 256, 8 * ptq::kProbeBoxBytes, s>>>(tm0, m_tiles, N / 256);
+                break;
+            case ptq::kProbeOperandPull:
+                ptq::ptq_probe_operand_pull_kernel<<<sms, 64, 4 * ptq::kProbeStageBytes + 128, s>>>(tm0, tm1, m_tiles, N / 256, K / 128, status);
+                break;
+            case ptq::kProbeLaunch:
+                ptq::ptq_probe_empty_kernel<<<sms, 256, 0, s>>>(0);
+                break;
+            default:
+                return launch_pdl(ptq::ptq_probe_empty_kernel, sms, 256, 0, s, 1);
+        }
+        return cudaGetLastError();
+    };
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    PTQ_CUDA(cudaEventCreate(&e0));
+    cudaError_t err = cudaEventCreate(&e1);
+    for (int i = 0; i < 3 && err == cudaSuccess; ++i) err = launch();
+    if (err == cudaSuccess) err = cudaEventRecord(e0, s);
+    for (int i = 0; i < iters && err == cudaSuccess; ++i) err = launch();
+    if (err == cudaSuccess) err = cudaEventRecord(e1, s);
+    if (err == cudaSuccess) err = cudaEventSynchronize(e1);
+    float ms = 0.0f;
+    if (err == cudaSuccess) err = cudaEventElapsedTime(&ms, e0, e1);
+    g_launches.fetch_add(static_cast<unsigned long long>(iters) + 3ull, std::memory_order_relaxed);
+    cudaEventDestroy(e0);
+    if (e1) cudaEventDestroy(e1);
+    if (err != cudaSuccess) return fail(PTQ_ERR_CUDA, "probe: %s", cudaGetErrorString(err));
+    if (status) {
+        unsigned word = 0;
+        PTQ_CUDA(cudaMemcpy(&word, status, sizeof(word), cudaMemcpyDeviceToHost));
+        if (word) return fail(PTQ_ERR_TIMEOUT, "probe: a bounded wait gave up (status word 0x%x)", word);
+    }
+    const double per_launch_s = static_cast<double>(ms) * 1e-3 / iters;
+    *result = moves_bytes ? moved / per_launch_s / 1e9 : per_launch_s * 1e6;   // GB/s, or microseconds per launch
+    return PTQ_OK;
 }
 
 static ptq_status_t calibrate_impl(int K, int N, int T, const void *xcal_fp16, int Bc, const int8_t *w_q,

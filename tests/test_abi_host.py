@@ -74,6 +74,12 @@ def test_null_handles_are_refused_not_dereferenced(lib):
     assert lib.ptq_linear_workspace_bytes(None, 4, 0) == 0
     assert lib.ptq_linear_fused_supported(None) == 0
     assert lib.ptq_linear_gemm_variant(None, 1) == -1
+    out = ctypes.c_double(-1.0)
+    assert lib.ptq_probe(0, None, 0, 10, None, None) == 1                      # PTQ_ERR_NULL: no result pointer
+    assert lib.ptq_probe(9, None, 0, 10, ctypes.byref(out), None) == 3         # PTQ_ERR_VALUE: unknown kind
+    assert lib.ptq_probe(0, None, 0, 0, ctypes.byref(out), None) == 3          # iters out of range
+    assert lib.ptq_probe(1, None, 1 << 20, 10, ctypes.byref(out), None) == 1   # a byte-moving kind needs a buffer
+    assert out.value == 0.0
     assert lib.ptq_linear_forward(None, None, 1, None, None, 0, 0, None) == 1
     assert lib.ptq_quantize(None, None, 1, None, None) == 1
     assert lib.ptq_linear_device_status(None) == 1

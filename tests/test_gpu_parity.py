@@ -361,3 +361,26 @@ def test_gemm_kernel_selection_covers_all_three_variants(env):
         layer = ptq.PtqLinear(wq, dw, s, dx, bias)
         assert layer.gemm_variant(spec.B) == variant, (spec.name, spec.M, spec.K, spec.N, layer.gemm_variant(spec.B))
         assert layer.gemm_variant(0) == -1
+
+
+def test_probe_kernels_report_plausible_rates(env):
+    """The measurement aids behind the roofline discussion: on a B200 a pure store stream and TMA stores in the
+    epilogue's pattern both exceed 3 TB/s, operand stages arrive from L2 faster than the stores leave, and an empty
+    kernel launches in microseconds.  Small buffers and bad arguments are refused, and nothing is left in flight."""
+    ptq, torch = env
+    P = ptq.binding
+    buf = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    st16 = P.probe(P.PROBE_STORE16, buf, 5)
+    tma = P.probe(P.PROBE_TMA_STORE, buf, 5)
+    pull = P.probe(P.PROBE_OPERAND_PULL, buf[:64 << 20], 5)
+    assert 3000.0 < st16 < 12000.0 and 3000.0 < tma < 12000.0, (st16, tma)
+    assert pull > tma and pull < 60000.0, pull
+    assert 0.5 < P.probe(P.PROBE_LAUNCH_PDL, None, 200) < 50.0
+    assert 0.5 < P.probe(P.PROBE_LAUNCH, None, 200) < 50.0
+    with pytest.raises(ptq.PtqError) as e:
+        P.probe(P.PROBE_TMA_STORE, buf[:1024], 5)
+    assert e.value.status == 2
+    with pytest.raises(ptq.PtqError) as e:
+        P.probe(P.PROBE_STORE16, buf[64:], 5)                       # not 256-byte aligned
+    assert e.value.status == 4
+    torch.cuda.synchronize()
