@@ -305,6 +305,8 @@ ptq_status_t launch_quantize(const ptq_linear *h, const void *x, long long M, vo
     }
     p.B = static_cast<int>(B);
     p.imgs_per_iter = static_cast<int>(S);
+    p.fd_cpi = ptq::make_fastdiv(static_cast<unsigned>(vec ? cpi : 1));
+    p.fd_cpr = ptq::make_fastdiv(static_cast<unsigned>(vec ? h->K / 8 : 1));
     if (vec) {
         const int grid = static_cast<int>(S * cpi / 256);
         if (h->act_bits == 4) {

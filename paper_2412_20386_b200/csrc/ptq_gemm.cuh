@@ -67,26 +67,6 @@ constexpr int kGemmSmemBytes = gemm_smem_bytes(kStages, 1, 0);
 static_assert(kGemmSmemBytes <= 232448 && gemm_smem_bytes(kStages - 1, 2, 1) <= kGemmSmemBytes,
               "streaming GEMM kernel exceeds the shared memory of one CTA");
 
-// Division of a 32-bit number by a launch constant without a division: with magic = ceil(2^64 / d), the
-// high 64 bits of magic * n are floor(n / d) for every 32-bit n.  A runtime integer division is a chain of
-// some twenty dependent instructions; at the top of an epilogue loop, where the warp has nothing else to
-// issue, several of them cost hundreds of cycles per tile.
-struct FastDiv {
-    unsigned d;
-    unsigned long long magic;
-};
-__host__ __device__ inline FastDiv make_fastdiv(unsigned d)
-{
-    FastDiv f;
-    f.d = d;
-    f.magic = d > 1u ? 0xFFFFFFFFFFFFFFFFull / d + 1ull : 0ull;
-    return f;
-}
-__device__ __forceinline__ unsigned fd_div(unsigned n, const FastDiv &f)
-{
-    return f.d == 1u ? n : static_cast<unsigned>(__umul64hi(f.magic, static_cast<unsigned long long>(n)));
-}
-
 struct GemmParams {
     long long M;
     int N, K, T;

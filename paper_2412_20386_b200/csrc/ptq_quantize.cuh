@@ -219,6 +219,7 @@ struct QuantParams {
     int q_pitch;         // bytes between rows of q
     int B;               // images (M = B * T)
     int imgs_per_iter;   // vector kernel: images between consecutive chunks of one thread
+    FastDiv fd_cpi, fd_cpr;   // vector kernel: divisors T * K / 8 (chunks per image) and K / 8 (chunks per row)
 };
 
 #ifndef PTQ_QUANT_CTAS_PER_SM
@@ -275,10 +276,12 @@ __global__ void __launch_bounds__(256, kQuantCtasPerSm) ptq_quantize_vec8_kernel
     __shared__ uint4 ring[D][256];
     const int cpr = p.K >> 3;                                        // chunks per row
     const int cpi = p.T * cpr;                                       // chunks per image
-    const long long gtid = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
-    const int c = static_cast<int>(gtid % cpi);
-    int b = static_cast<int>(gtid / cpi);
-    const int t = c / cpr;
+    // the grid is at most four resident waves, so the global thread index fits 32 bits; no runtime divisions
+    // in front of the parameter loads below (a CTA that starts late runs this prologue on the critical path)
+    const unsigned gtid = blockIdx.x * blockDim.x + threadIdx.x;
+    int b = static_cast<int>(fd_div(gtid, p.fd_cpi));
+    const int c = static_cast<int>(gtid) - b * cpi;
+    const int t = static_cast<int>(fd_div(static_cast<unsigned>(c), p.fd_cpr));
     const int kc = c - t * cpr;
     const int S = p.imgs_per_iter;
 
@@ -286,12 +289,13 @@ __global__ void __launch_bounds__(256, kQuantCtasPerSm) ptq_quantize_vec8_kernel
     const int z = kMode == kCodeU8 ? __ldg(p.zp + t) : 0;
     const float *s8 = p.s + kc * 8;          // read only on the exact route
     const float *rs8 = p.rs + kc * 8;
-    float c8[8];
+    // The parameter loads are issued here, in front of the dependency wait, but their values are first used after
+    // the ring has been filled: a CTA that starts late (its wait is already satisfied) then has the parameter
+    // loads and its first activation loads in flight together instead of one memory latency after the other.
+    float4 r0 = make_float4(0.0f, 0.0f, 0.0f, 0.0f), r1 = r0;
     if (kFast) {
-        const float4 r0 = __ldg(reinterpret_cast<const float4 *>(rs8));
-        const float4 r1 = __ldg(reinterpret_cast<const float4 *>(rs8) + 1);
-        c8[0] = __fmul_rn(r0.x, d.y); c8[1] = __fmul_rn(r0.y, d.y); c8[2] = __fmul_rn(r0.z, d.y); c8[3] = __fmul_rn(r0.w, d.y);
-        c8[4] = __fmul_rn(r1.x, d.y); c8[5] = __fmul_rn(r1.y, d.y); c8[6] = __fmul_rn(r1.z, d.y); c8[7] = __fmul_rn(r1.w, d.y);
+        r0 = __ldg(reinterpret_cast<const float4 *>(rs8));
+        r1 = __ldg(reinterpret_cast<const float4 *>(rs8) + 1);
     }
 
     const long long x_img = static_cast<long long>(p.T) * p.K;          // elements per image of x
@@ -309,6 +313,11 @@ __global__ void __launch_bounds__(256, kQuantCtasPerSm) ptq_quantize_vec8_kernel
     for (int i = 0; i < D; ++i) {
         if (b + i * S < p.B) cp_async_16(&ring[i][threadIdx.x], xp + i * x_step);
         cp_async_commit();
+    }
+    float c8[8];
+    if (kFast) {
+        c8[0] = __fmul_rn(r0.x, d.y); c8[1] = __fmul_rn(r0.y, d.y); c8[2] = __fmul_rn(r0.z, d.y); c8[3] = __fmul_rn(r0.w, d.y);
+        c8[4] = __fmul_rn(r1.x, d.y); c8[5] = __fmul_rn(r1.y, d.y); c8[6] = __fmul_rn(r1.z, d.y); c8[7] = __fmul_rn(r1.w, d.y);
     }
     int slot = 0;
     while (b < p.B) {

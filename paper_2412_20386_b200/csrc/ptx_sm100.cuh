@@ -27,6 +27,27 @@ __device__ __forceinline__ unsigned long long global_timer_ns()
     return t;
 }
 
+// ---------------------------------------------------------------- integer division by launch constants
+// Division of a 32-bit number by a launch constant without a division: with magic = ceil(2^64 / d), the
+// high 64 bits of magic * n are floor(n / d) for every 32-bit n.  A runtime integer division is a chain of
+// some twenty dependent instructions (far more for 64-bit operands); at the top of an epilogue loop or in a
+// kernel's prologue, where the warp has nothing else to issue, several of them cost hundreds of cycles.
+struct FastDiv {
+    unsigned d;
+    unsigned long long magic;
+};
+__host__ __device__ inline FastDiv make_fastdiv(unsigned d)
+{
+    FastDiv f;
+    f.d = d;
+    f.magic = d > 1u ? 0xFFFFFFFFFFFFFFFFull / d + 1ull : 0ull;
+    return f;
+}
+__device__ __forceinline__ unsigned fd_div(unsigned n, const FastDiv &f)
+{
+    return f.d == 1u ? n : static_cast<unsigned>(__umul64hi(f.magic, static_cast<unsigned long long>(n)));
+}
+
 // ---------------------------------------------------------------- mbarrier
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
 {
