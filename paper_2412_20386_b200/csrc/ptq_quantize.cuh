@@ -231,10 +231,21 @@ struct QuantParams {
 constexpr int kQuantCtasPerSm = PTQ_QUANT_CTAS_PER_SM;   // resident CTAs per SM the vector kernel is built and launched for
 constexpr int kQuantRingDepth = PTQ_QUANT_RING_DEPTH;    // 16-byte loads in flight per thread
 
-__device__ __forceinline__ void cp_async_16(void *smem_dst, const void *gmem_src)
+// L2 cache policy of the quantize kernel's loads: the activations are read once and never again, so they are
+// marked evict-first and do not push the codes (read back by the GEMM kernel launched next) or the next layer's
+// parameters out of L2.  Measured: the K = 768 layer of Vim-B 21.3 -> 20.4 us, nothing else changes.  Marking the
+// code stores evict-last as well made the GEMM kernels of small-K layers 6 % faster when timed alone, but the
+// Vim-B in_proj GEMM 4 % slower and no step faster, so the stores keep the default policy.
+__device__ __forceinline__ uint64_t l2_policy_evict_first()
+{
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ void cp_async_16_hint(void *smem_dst, const void *gmem_src, uint64_t policy)
 {
     const unsigned d = static_cast<unsigned>(__cvta_generic_to_shared(smem_dst));
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gmem_src) : "memory");
+    asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;" ::"r"(d), "l"(gmem_src), "l"(policy) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
@@ -308,10 +319,11 @@ __global__ void __launch_bounds__(256, kQuantCtasPerSm) ptq_quantize_vec8_kernel
     griddep_wait();
     griddep_launch_dependents();
 
+    const uint64_t pol_x = l2_policy_evict_first();
     // fill the ring: slot i holds image b + i*S (one commit group per slot, empty past the last image)
 #pragma unroll
     for (int i = 0; i < D; ++i) {
-        if (b + i * S < p.B) cp_async_16(&ring[i][threadIdx.x], xp + i * x_step);
+        if (b + i * S < p.B) cp_async_16_hint(&ring[i][threadIdx.x], xp + i * x_step, pol_x);
         cp_async_commit();
     }
     float c8[8];
@@ -325,7 +337,7 @@ __global__ void __launch_bounds__(256, kQuantCtasPerSm) ptq_quantize_vec8_kernel
         const uint4 v = ring[slot][threadIdx.x];
         *reinterpret_cast<uint2 *>(qp) = quantize8<kFast, kMode>(v, c8, s8, rs8, d.x, d.y, z);
         // refill the slot just consumed (its value has been used above) with the image D*S further on
-        if (b + D * S < p.B) cp_async_16(&ring[slot][threadIdx.x], xp + D * x_step);
+        if (b + D * S < p.B) cp_async_16_hint(&ring[slot][threadIdx.x], xp + D * x_step, pol_x);
         cp_async_commit();
         slot = (slot + 1 == D) ? 0 : slot + 1;
         b += S;
