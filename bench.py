@@ -626,8 +626,8 @@ def run_ours(args, specs, rank, world, local_rank):
 TRAFFIC = {
     ("ptq_gemm_dequant_panel_kernel", "c3", "in_proj"): 41.260032e6 + 250.792704e6,
     ("ptq_gemm_dequant_kernel", "c3", "out_proj"): 78.710528e6 + 32.977152e6,
-    ("ptq_quantize_kernel", "c3", "in_proj"): 77.504000e6 + 10.326528e6,
-    ("ptq_quantize_kernel", "c3", "out_proj"): 155.117824e6 + 45.882624e6,
+    ("ptq_quantize_kernel", "c3", "in_proj"): 77.492224e6 + 6.748672e6,
+    ("ptq_quantize_kernel", "c3", "out_proj"): 155.017472e6 + 22.338304e6,
 }
 
 
