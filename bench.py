@@ -624,8 +624,8 @@ def run_ours(args, specs, rank, world, local_rank):
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised
 # under profiles/; keyed by (kernel, workload, layer).  An entry is removed when its kernel changes.
 TRAFFIC = {
-    ("ptq_gemm_dequant_panel_kernel", "c3", "in_proj"): 41.260032e6 + 250.792704e6,
-    ("ptq_gemm_dequant_kernel", "c3", "out_proj"): 78.710528e6 + 32.977152e6,
+    ("ptq_gemm_dequant_panel_kernel", "c3", "in_proj"): 41.190144e6 + 250.822144e6,
+    ("ptq_gemm_dequant_kernel", "c3", "out_proj"): 78.705408e6 + 33.518592e6,
     ("ptq_quantize_kernel", "c3", "in_proj"): 77.492224e6 + 6.748672e6,
     ("ptq_quantize_kernel", "c3", "out_proj"): 155.017472e6 + 22.338304e6,
 }
