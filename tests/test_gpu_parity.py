@@ -193,6 +193,22 @@ def test_odd_shapes_and_ragged_tiles(env, K, N, T, B):
     check_layer(ptq, torch, spec)
 
 
+@pytest.mark.parametrize("K,N,T,B,variant", [(520, 600, 197, 257, 2),      # panel kernel: ragged K, N and M tails, 5 k-blocks
+                                             (776, 1032, 64, 300, 0),     # 7 k-blocks: too deep for a panel, streaming
+                                             (72, 520, 197, 140, 1)])     # two-team epilogue: ragged K and N, 3 N tiles
+def test_ragged_shapes_through_the_panel_and_team_kernels(env, K, N, T, B, variant):
+    """Shapes chosen so that the resident-panel kernel and the two-team epilogue (and, as a control, the streaming
+    kernel at the same size) see tails in every dimension: K not a multiple of 128, N not a multiple of the tile
+    width, B*T not a multiple of 128, an uneven last round of work units."""
+    ptq, torch = env
+    spec = wl.LinearSpec(10, K % 89, N % 7, "ragged", B, T, K, N, bias=False)
+    x, wq, dw, bias, s, dx = layer_inputs(spec, B=1)
+    layer = ptq.PtqLinear(wq, dw, s, dx, bias)
+    assert layer.gemm_variant(B) == variant
+    layer.close()
+    check_layer(ptq, torch, spec, flags_list=(0,))
+
+
 def test_seeded_random_shapes(env):
     """Sixteen seeded random (K, N, T, B): every kernel variant the shape and alignment select, every flag."""
     ptq, torch = env
