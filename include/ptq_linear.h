@@ -127,7 +127,8 @@ size_t ptq_linear_workspace_bytes(const ptq_linear_t *h, int B, unsigned flags);
  *   y_fp16     device, [B,T,N] contiguous binary16; must not overlap x or the workspace
  *   workspace  device, at least ptq_linear_workspace_bytes(h,B,flags) bytes, 16-byte aligned;
  *              contents are scratch.  May be NULL with PTQ_FLAG_FUSED_PROLOGUE.
- *   flags      PTQ_FLAG_NONE: quantize kernel, then GEMM+dequant kernel.
+ *   flags      PTQ_FLAG_NONE: quantize kernel, then GEMM+dequant kernel (one of three variants chosen from
+ *              the shape, all with the same bits: see ptq_linear_gemm_variant).
  *              PTQ_FLAG_FUSED_PROLOGUE: one kernel; same results bit for bit.  Layers whose shape the
  *              fused kernel does not cover fall back to the two-kernel path and then need the workspace
  *              (ptq_linear_fused_supported tells which).
