@@ -209,6 +209,47 @@ def test_ragged_shapes_through_the_panel_and_team_kernels(env, K, N, T, B, varia
     check_layer(ptq, torch, spec, flags_list=(0,))
 
 
+def test_two_host_threads_share_one_handle(env):
+    """Two host threads call forward on ONE handle at the same time, each on its own stream with its own buffers
+    (ctypes releases the interpreter lock during the call, so the library's per-handle caches and one-time set-up
+    are really entered concurrently).  Every output must equal the single-threaded one bit for bit."""
+    import threading
+    ptq, torch = env
+    spec = CFG[1][0]
+    x, wq, dw, bias, s, dx = layer_inputs(spec, B=8)
+    layer = ptq.PtqLinear(wq, dw, s, dx, bias)
+    xd = torch.from_numpy(x).cuda()
+    want = layer.forward(xd)
+    torch.cuda.synchronize()
+    outs, errors = {}, []
+
+    def worker(tid):
+        try:
+            torch.cuda.set_device(0)
+            st = torch.cuda.Stream()
+            xs = xd.clone()
+            ys = [torch.empty_like(want) for _ in range(6)]          # more buffers than cache entries
+            ws = torch.empty(layer.workspace_bytes(8), dtype=torch.uint8, device="cuda")
+            torch.cuda.synchronize()
+            for i in range(60):
+                layer.forward(xs, y=ys[i % 6], workspace=ws, stream=st)
+            st.synchronize()
+            outs[tid] = ys
+        except Exception as e:                                        # noqa: BLE001 (reported below)
+            errors.append(e)
+
+    threads = [threading.Thread(target=worker, args=(t,)) for t in range(2)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
+    layer.device_status()
+    for ys in outs.values():
+        for y in ys:
+            assert torch.equal(y, want)
+
+
 def test_seeded_random_shapes(env):
     """Sixteen seeded random (K, N, T, B): every kernel variant the shape and alignment select, every flag."""
     ptq, torch = env
